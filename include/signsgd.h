@@ -1,0 +1,156 @@
+/*
+ * signsgd.h -- C ABI of the B200 (sm_100a) library for the data-parallel hot path of
+ * signSGD / Signum with majority vote (Algorithm 1 of "signSGD with Majority Vote is
+ * Communication Efficient and Fault Tolerant").
+ *
+ * One iteration of Algorithm 1, for M workers whose gradients sit in one GPU's memory:
+ *
+ *   on worker m:   v_m <- (1 - beta) g_m + beta v_m          ("update momentum")
+ *                  push sign(v_m)                             (1 bit per coordinate)
+ *   on server:     V <- sum_m sign(v_m);  push sign(V)        ("majority vote")
+ *   on every worker: x <- x - eta (sign(V) + lambda x)        ("update parameters")
+ *
+ * Conventions shared by every entry point
+ * ---------------------------------------
+ * Sign code.   sign(z) is carried in one bit: bit = 1 means +1, and bit = 1 iff z >= 0 as a
+ *              value (+0.0 and -0.0 give 1, NaN gives 0, +Inf gives 1, -Inf gives 0). The
+ *              vote uses the same rule on the integer tally V, so a tie at even M votes +1.
+ * Packing.     d coordinates occupy W = ceil(d/32) uint32 words (the 32x compression of the
+ *              abstract). Coordinate 32 j + i is bit i of word j, bit 0 least significant.
+ *              Bits at coordinates >= d are written as 0 in every output.
+ * Arithmetic.  fp32, round to nearest even, every multiply and add rounded separately (no
+ *              fused multiply-add), denormals kept. (1 - beta) is formed once in fp32 on the
+ *              host. bf16 gradients are widened exactly to fp32. With weight_decay == 0 the
+ *              update is x <- x - (+-lr); otherwise x <- x - lr * (s + weight_decay * x) with
+ *              s = +-1, evaluated in that order.
+ * Adversaries. flip_mask bit m set makes worker m an inverting adversary (Definition 1 (iii),
+ *              Section 4.2): its sign bits are complemented before the vote. Bits >= M must be 0.
+ * Memory.      Every data buffer is caller-owned DEVICE memory unless a parameter is documented
+ *              as host memory. Arrays of pointers (grads, momenta, packed) are HOST arrays of M
+ *              device pointers; they are read during the call and may be freed after it returns.
+ *              The library allocates no device memory and never frees or keeps a caller pointer.
+ *              Buffers must not overlap each other; momentum and param are updated in place.
+ * Alignment.   Word buffers: 4 bytes. Gradients: their element size. fp32 state: 4 bytes. When
+ *              every gradient, momentum and parameter pointer of a call is 16-byte aligned
+ *              (8-byte for bf16 gradients) the 128-bit vectorised kernels run; otherwise a
+ *              scalar-load kernel with identical results runs. Misalignment below the element
+ *              size is SS_ERR_MISALIGNED.
+ * Streams.     cuda_stream is a cudaStream_t (NULL = the legacy default stream). Calls enqueue
+ *              work on it and return without synchronising. The device that is current when
+ *              the call is made is used.
+ * Limits.      1 <= M <= SS_MAX_WORKERS. d >= 0; d == 0 is a no-op that returns SS_OK.
+ * Errors.      Every function returns an int status: SS_OK (0) or a negative SS_ERR_* code;
+ *              nothing is thrown across the boundary. On an argument error nothing is enqueued.
+ *              SS_ERR_CUDA reports a failed launch or runtime call; ss_last_cuda_error() gives
+ *              its cudaError_t value for the calling thread.
+ */
+#ifndef SIGNSGD_H_
+#define SIGNSGD_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define SS_MAX_WORKERS 64
+
+typedef enum { SS_F32 = 0, SS_BF16 = 1 } ss_dtype;
+
+enum {
+    SS_OK = 0,
+    SS_ERR_INVALID_ARG = -1,  /* NULL pointer, M or d out of range, flip_mask bit >= M, bad dtype */
+    SS_ERR_MISALIGNED = -2,   /* pointer not aligned to its element size */
+    SS_ERR_UNSUPPORTED = -3,  /* valid request that this build cannot serve */
+    SS_ERR_CUDA = -4          /* CUDA runtime or launch failure */
+};
+
+/* ceil(d/32): words needed for d sign bits (abstract: 32x less than fp32). -1 if d < 0. */
+int64_t ss_packed_words(int64_t d);
+
+/* Static, human-readable name of a status code. Never NULL. */
+const char* ss_status_string(int status);
+
+/* cudaError_t of the last SS_ERR_CUDA returned on the calling thread (0 if none). */
+int ss_last_cuda_error(void);
+
+/*
+ * Sign compression of one worker's gradient (Algorithm 1, "push sign(.)" with beta = 0;
+ * Section 4: bit-packing a sign tensor to one bit per element).
+ *   grad       in   d elements of dtype dt
+ *   out_words  out  ceil(d/32) words
+ */
+int ss_sign_pack(const void* grad, ss_dtype dt, int64_t d, uint32_t* out_words, void* cuda_stream);
+
+/*
+ * Server side of Algorithm 1: V = sum_m sign(v_m), result sign(V), on packed words.
+ *   packed      in   HOST array of M device pointers, each to ceil(d/32) words
+ *   vote_words  out  ceil(d/32) words; must not overlap any input
+ * Bits of the inputs at coordinates >= d are ignored.
+ */
+int ss_majority_vote(const uint32_t* const* packed, int M, int64_t d, uint64_t flip_mask,
+                     uint32_t* vote_words, void* cuda_stream);
+
+/*
+ * Worker side of Algorithm 1 with momentum: v <- (1 - beta) g + beta v in place, then sign(v)
+ * packed. beta = 0 gives the packed sign of g (and v = g).
+ *   grad       in      d elements of dtype dt
+ *   momentum   in/out  d fp32
+ *   out_words  out     ceil(d/32) words
+ */
+int ss_signum_update(const void* grad, ss_dtype dt, float* momentum, float beta, int64_t d,
+                     uint32_t* out_words, void* cuda_stream);
+
+/*
+ * Algorithm 1, "update parameters": x <- x - lr (sign(V) + weight_decay x) from the packed vote.
+ *   param       in/out  d fp32
+ *   vote_words  in      ceil(d/32) words
+ */
+int ss_apply_vote(float* param, const uint32_t* vote_words, int64_t d, float lr,
+                  float weight_decay, void* cuda_stream);
+
+/*
+ * One whole iteration of Algorithm 1 in a single pass over memory: momentum, sign, vote and
+ * parameter update per coordinate, the packed signs never leaving the chip.
+ *   grads           in      HOST array of M device pointers, d elements of dt each
+ *   momenta         in/out  HOST array of M device pointers to d fp32 each, or NULL for
+ *                           signSGD (no momentum state; beta is ignored)
+ *   param           in/out  d fp32
+ *   vote_words_out  out     ceil(d/32) words, or NULL if the packed vote is not wanted
+ * Results are identical, bit for bit, to ss_signum_update (or ss_sign_pack) per worker followed
+ * by ss_majority_vote and ss_apply_vote.
+ */
+int ss_fused_step(const void* const* grads, ss_dtype dt, float* const* momenta, int M, int64_t d,
+                  float beta, uint64_t flip_mask, float* param, float lr, float weight_decay,
+                  uint32_t* vote_words_out, void* cuda_stream);
+
+/*
+ * ss_fused_step for gradients that start in HOST memory (the end-to-end form: what a step costs
+ * when the M gradients arrive over PCIe and the packed vote goes back, as the d-bit messages of
+ * Algorithm 1's push steps do).
+ *   host_grads      in      HOST array of M HOST pointers (pinned memory recommended), d elements each
+ *   staging         scratch HOST array of M device pointers, d elements of dt each; overwritten
+ *   momenta, param, M, d, beta, flip_mask, lr, weight_decay: as ss_fused_step (device memory)
+ *   vote_words_dev  out     ceil(d/32) words of device memory (required)
+ *   host_vote_out   out     ceil(d/32) words of HOST memory, or NULL to skip the copy back
+ * Enqueues M host-to-device copies, the fused kernel and one device-to-host copy on cuda_stream
+ * and returns; host_grads and host_vote_out must stay valid until the stream has drained.
+ */
+int ss_fused_step_host(const void* const* host_grads, ss_dtype dt, void* const* staging,
+                       float* const* momenta, int M, int64_t d, float beta, uint64_t flip_mask,
+                       float* param, float lr, float weight_decay, uint32_t* vote_words_dev,
+                       uint32_t* host_vote_out, void* cuda_stream);
+
+/*
+ * Launch-shape override for benchmarking sweeps (process-wide; not part of the method).
+ *   key: "threads" (block size, multiple of 32 in [64, 1024], 0 = default) or
+ *        "blocks_per_sm" (persistent blocks per SM, 0 = as many as fit).
+ * Returns SS_ERR_INVALID_ARG for an unknown key or a value out of range.
+ */
+int ss_set_launch_option(const char* key, int value);
+
+#ifdef __cplusplus
+}
+#endif
+
+#endif /* SIGNSGD_H_ */

@@ -1,0 +1,221 @@
+"""Python names for the C ABI of libsignsgd.so -- argument marshalling only.
+
+Each function below has the name and the argument order of its C entry point (see
+``include/signsgd.h``) and does nothing but check tensor types, take ``data_ptr()`` and the
+current CUDA stream, call into the library and raise on a non-zero status. All arithmetic
+of Algorithm 1 happens in the CUDA kernels. There is no CPU fallback: if the library has
+not been built (``python -m paper_1810_05291_b200.build``), the first call raises.
+
+Tensors: gradients ``float32`` or ``bfloat16``; momenta and parameters ``float32``; packed
+signs and votes ``int32`` (bit pattern of the uint32 words), ``ceil(d/32)`` of them.
+"""
+
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional, Sequence
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libsignsgd.so")
+
+SS_F32 = 0
+SS_BF16 = 1
+SS_MAX_WORKERS = 64
+
+SS_OK = 0
+SS_ERR_INVALID_ARG = -1
+SS_ERR_MISALIGNED = -2
+SS_ERR_UNSUPPORTED = -3
+SS_ERR_CUDA = -4
+
+EXPORTS = ("ss_packed_words", "ss_status_string", "ss_last_cuda_error", "ss_sign_pack",
+           "ss_majority_vote", "ss_signum_update", "ss_apply_vote", "ss_fused_step",
+           "ss_fused_step_host", "ss_set_launch_option")
+
+_lib = None
+
+
+class SignSGDError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        msg = lib().ss_status_string(status).decode()
+        if status == SS_ERR_CUDA:
+            msg += " [cudaError %d]" % lib().ss_last_cuda_error()
+        super().__init__("%s: %s" % (where, msg))
+
+
+def lib() -> ctypes.CDLL:
+    """Load libsignsgd.so (once). Raises if it has not been built: there is no fallback."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise RuntimeError(
+            "libsignsgd.so is missing (%s). Build it with `python -m paper_1810_05291_b200.build`; "
+            "this package has no CPU or PyTorch fallback." % LIB_PATH)
+    L = ctypes.CDLL(LIB_PATH)
+    vp, i64, i32, u64, f32 = (ctypes.c_void_p, ctypes.c_int64, ctypes.c_int, ctypes.c_uint64,
+                              ctypes.c_float)
+    L.ss_packed_words.argtypes = [i64]
+    L.ss_packed_words.restype = i64
+    L.ss_status_string.argtypes = [i32]
+    L.ss_status_string.restype = ctypes.c_char_p
+    L.ss_last_cuda_error.argtypes = []
+    L.ss_last_cuda_error.restype = i32
+    L.ss_sign_pack.argtypes = [vp, i32, i64, vp, vp]
+    L.ss_majority_vote.argtypes = [vp, i32, i64, u64, vp, vp]
+    L.ss_signum_update.argtypes = [vp, i32, vp, f32, i64, vp, vp]
+    L.ss_apply_vote.argtypes = [vp, vp, i64, f32, f32, vp]
+    L.ss_fused_step.argtypes = [vp, i32, vp, i32, i64, f32, u64, vp, f32, f32, vp, vp]
+    L.ss_fused_step_host.argtypes = [vp, i32, vp, vp, i32, i64, f32, u64, vp, f32, f32, vp, vp, vp]
+    L.ss_set_launch_option.argtypes = [ctypes.c_char_p, i32]
+    for name in ("ss_sign_pack", "ss_majority_vote", "ss_signum_update", "ss_apply_vote",
+                 "ss_fused_step", "ss_fused_step_host", "ss_set_launch_option"):
+        getattr(L, name).restype = i32
+    _lib = L
+    return L
+
+
+# ---- marshalling helpers ------------------------------------------------------------------
+
+def _dtype_code(t: torch.Tensor) -> int:
+    if t.dtype == torch.float32:
+        return SS_F32
+    if t.dtype == torch.bfloat16:
+        return SS_BF16
+    raise TypeError("gradient dtype must be float32 or bfloat16, got %s" % t.dtype)
+
+
+def _dev(t: torch.Tensor, dtype, name: str, n: Optional[int] = None) -> int:
+    if not t.is_cuda:
+        raise ValueError("%s must be a CUDA tensor" % name)
+    if dtype is not None and t.dtype != dtype:
+        raise TypeError("%s must be %s, got %s" % (name, dtype, t.dtype))
+    if t.dim() != 1 or not t.is_contiguous():
+        raise ValueError("%s must be a contiguous 1-D tensor" % name)
+    if n is not None and t.numel() != n:
+        raise ValueError("%s must have %d elements, has %d" % (name, n, t.numel()))
+    return t.data_ptr()
+
+
+def _words(t: torch.Tensor, d: int, name: str) -> int:
+    return _dev(t, torch.int32, name, ss_packed_words(d))
+
+
+def _ptr_array(ptrs: Sequence[int]):
+    return (ctypes.c_void_p * len(ptrs))(*ptrs)
+
+
+def _stream(stream) -> ctypes.c_void_p:
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return ctypes.c_void_p(stream.cuda_stream if hasattr(stream, "cuda_stream") else int(stream))
+
+
+def _check(status: int, where: str) -> None:
+    if status != SS_OK:
+        raise SignSGDError(status, where)
+
+
+# ---- the entry points -----------------------------------------------------------------------
+
+def ss_packed_words(d: int) -> int:
+    return int(lib().ss_packed_words(int(d)))
+
+
+def ss_status_string(status: int) -> str:
+    return lib().ss_status_string(int(status)).decode()
+
+
+def ss_set_launch_option(key: str, value: int) -> None:
+    _check(lib().ss_set_launch_option(key.encode(), int(value)), "ss_set_launch_option")
+
+
+def ss_sign_pack(grad: torch.Tensor, out_words: torch.Tensor, stream=None) -> None:
+    d = grad.numel()
+    _check(lib().ss_sign_pack(_dev(grad, None, "grad"), _dtype_code(grad), d,
+                              _words(out_words, d, "out_words"), _stream(stream)), "ss_sign_pack")
+
+
+def ss_majority_vote(packed: Sequence[torch.Tensor], d: int, flip_mask: int,
+                     vote_words: torch.Tensor, stream=None) -> None:
+    ptrs = [_words(p, d, "packed[%d]" % m) for m, p in enumerate(packed)]
+    _check(lib().ss_majority_vote(_ptr_array(ptrs), len(ptrs), int(d), int(flip_mask),
+                                  _words(vote_words, d, "vote_words"), _stream(stream)),
+           "ss_majority_vote")
+
+
+def ss_signum_update(grad: torch.Tensor, momentum: torch.Tensor, beta: float,
+                     out_words: torch.Tensor, stream=None) -> None:
+    d = grad.numel()
+    _check(lib().ss_signum_update(_dev(grad, None, "grad"), _dtype_code(grad),
+                                  _dev(momentum, torch.float32, "momentum", d), float(beta), d,
+                                  _words(out_words, d, "out_words"), _stream(stream)),
+           "ss_signum_update")
+
+
+def ss_apply_vote(param: torch.Tensor, vote_words: torch.Tensor, lr: float,
+                  weight_decay: float = 0.0, stream=None) -> None:
+    d = param.numel()
+    _check(lib().ss_apply_vote(_dev(param, torch.float32, "param"), _words(vote_words, d, "vote_words"),
+                               d, float(lr), float(weight_decay), _stream(stream)), "ss_apply_vote")
+
+
+def ss_fused_step(grads: Sequence[torch.Tensor], momenta: Optional[Sequence[torch.Tensor]],
+                  param: torch.Tensor, beta: float, lr: float, weight_decay: float = 0.0,
+                  flip_mask: int = 0, vote_words_out: Optional[torch.Tensor] = None,
+                  stream=None) -> None:
+    M = len(grads)
+    d = param.numel()
+    codes = {_dtype_code(g) for g in grads}
+    if len(codes) != 1:
+        raise TypeError("all gradients must share one dtype")
+    g_ptrs = [_dev(g, None, "grads[%d]" % m, d) for m, g in enumerate(grads)]
+    v_arr = None
+    if momenta is not None:
+        if len(momenta) != M:
+            raise ValueError("need one momentum buffer per worker")
+        v_arr = _ptr_array([_dev(v, torch.float32, "momenta[%d]" % m, d) for m, v in enumerate(momenta)])
+    w_ptr = None if vote_words_out is None else _words(vote_words_out, d, "vote_words_out")
+    _check(lib().ss_fused_step(_ptr_array(g_ptrs), codes.pop(), v_arr, M, d, float(beta),
+                               int(flip_mask), _dev(param, torch.float32, "param"), float(lr),
+                               float(weight_decay), w_ptr, _stream(stream)), "ss_fused_step")
+
+
+def ss_fused_step_host(host_grads: Sequence[torch.Tensor], staging: Sequence[torch.Tensor],
+                       momenta: Optional[Sequence[torch.Tensor]], param: torch.Tensor, beta: float,
+                       lr: float, weight_decay: float, flip_mask: int,
+                       vote_words_dev: torch.Tensor, host_vote_out: Optional[torch.Tensor],
+                       stream=None) -> None:
+    M = len(host_grads)
+    d = param.numel()
+    codes = {_dtype_code(g) for g in host_grads}
+    if len(codes) != 1:
+        raise TypeError("all gradients must share one dtype")
+    h_ptrs = []
+    for m, g in enumerate(host_grads):
+        if g.is_cuda or g.dim() != 1 or not g.is_contiguous() or g.numel() != d:
+            raise ValueError("host_grads[%d] must be a contiguous 1-D host tensor of d elements" % m)
+        h_ptrs.append(g.data_ptr())
+    if len(staging) != M:
+        raise ValueError("need one staging buffer per worker")
+    s_ptrs = [_dev(s, host_grads[0].dtype, "staging[%d]" % m, d) for m, s in enumerate(staging)]
+    v_arr = None
+    if momenta is not None:
+        if len(momenta) != M:
+            raise ValueError("need one momentum buffer per worker")
+        v_arr = _ptr_array([_dev(v, torch.float32, "momenta[%d]" % m, d) for m, v in enumerate(momenta)])
+    hv = None
+    if host_vote_out is not None:
+        if (host_vote_out.is_cuda or host_vote_out.dtype != torch.int32
+                or host_vote_out.numel() != ss_packed_words(d) or not host_vote_out.is_contiguous()):
+            raise ValueError("host_vote_out must be a contiguous host int32 tensor of ceil(d/32) words")
+        hv = host_vote_out.data_ptr()
+    _check(lib().ss_fused_step_host(_ptr_array(h_ptrs), codes.pop(), _ptr_array(s_ptrs), v_arr, M, d,
+                                    float(beta), int(flip_mask), _dev(param, torch.float32, "param"),
+                                    float(lr), float(weight_decay),
+                                    _words(vote_words_dev, d, "vote_words_dev"), hv, _stream(stream)),
+           "ss_fused_step_host")

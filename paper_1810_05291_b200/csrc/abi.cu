@@ -1,0 +1,228 @@
+// The C ABI: argument validation, alignment classification and kernel dispatch. Every step of
+// the path runs in the kernels; nothing here touches the data.
+#include <cstring>
+
+#include "common.cuh"
+
+namespace ss {
+
+LaunchOptions& launch_options() {
+    static LaunchOptions opts;
+    return opts;
+}
+
+int device_sm_count(cudaError_t* err) {
+    static int cached[64] = {0};
+    int dev = 0;
+    *err = cudaGetDevice(&dev);
+    if (*err != cudaSuccess) return 0;
+    if (dev >= 0 && dev < 64 && cached[dev] > 0) return cached[dev];
+    int sms = 0;
+    *err = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    if (*err != cudaSuccess) return 0;
+    if (dev >= 0 && dev < 64) cached[dev] = sms;
+    return sms;
+}
+
+namespace {
+
+thread_local int t_last_cuda_error = 0;
+
+int cuda_status(cudaError_t e) {
+    if (e == cudaSuccess) return SS_OK;
+    t_last_cuda_error = static_cast<int>(e);
+    return SS_ERR_CUDA;
+}
+
+inline bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) & (a - 1)) == 0; }
+
+inline int elem_bytes(ss_dtype dt) { return dt == SS_F32 ? 4 : 2; }
+
+inline bool dtype_ok(ss_dtype dt) { return dt == SS_F32 || dt == SS_BF16; }
+
+inline bool flip_ok(uint64_t flip, int M) { return M >= 64 || (flip >> M) == 0; }
+
+// half-open byte ranges [p, p + n)
+inline bool overlap(const void* p, size_t n, const void* q, size_t m) {
+    const uintptr_t a = reinterpret_cast<uintptr_t>(p), b = reinterpret_cast<uintptr_t>(q);
+    return n != 0 && m != 0 && a < b + m && b < a + n;
+}
+
+}  // namespace
+}  // namespace ss
+
+using namespace ss;
+
+extern "C" {
+#pragma GCC visibility push(default)
+
+int64_t ss_packed_words(int64_t d) { return d < 0 ? -1 : (d + 31) / 32; }
+
+const char* ss_status_string(int status) {
+    switch (status) {
+        case SS_OK: return "SS_OK";
+        case SS_ERR_INVALID_ARG: return "SS_ERR_INVALID_ARG: null pointer, size or worker count out of range, or flip_mask bit >= M";
+        case SS_ERR_MISALIGNED: return "SS_ERR_MISALIGNED: pointer not aligned to its element size";
+        case SS_ERR_UNSUPPORTED: return "SS_ERR_UNSUPPORTED: request not served by this build";
+        case SS_ERR_CUDA: return "SS_ERR_CUDA: CUDA runtime or launch failure (see ss_last_cuda_error)";
+        default: return "unknown status";
+    }
+}
+
+int ss_last_cuda_error(void) { return t_last_cuda_error; }
+
+int ss_set_launch_option(const char* key, int value) {
+    if (key == nullptr) return SS_ERR_INVALID_ARG;
+    if (std::strcmp(key, "threads") == 0) {
+        if (value != 0 && (value < 64 || value > 1024 || (value & 31) != 0)) return SS_ERR_INVALID_ARG;
+        launch_options().threads = value;
+        return SS_OK;
+    }
+    if (std::strcmp(key, "blocks_per_sm") == 0) {
+        if (value < 0 || value > 32) return SS_ERR_INVALID_ARG;
+        launch_options().blocks_per_sm = value;
+        return SS_OK;
+    }
+    return SS_ERR_INVALID_ARG;
+}
+
+static int step_common(const void* const* grads, ss_dtype dt, float* const* momenta, int M,
+                       int64_t d, float beta, uint64_t flip_mask, float* param, float lr,
+                       float weight_decay, uint32_t* words, void* cuda_stream) {
+    if (!dtype_ok(dt) || grads == nullptr || M < 1 || M > SS_MAX_WORKERS || d < 0) return SS_ERR_INVALID_ARG;
+    if (!flip_ok(flip_mask, M)) return SS_ERR_INVALID_ARG;
+    if (d == 0) return SS_OK;
+    if (param == nullptr && words == nullptr) return SS_ERR_INVALID_ARG;
+    const size_t eb = static_cast<size_t>(elem_bytes(dt));
+    const size_t gbytes = static_cast<size_t>(d) * eb, fbytes = static_cast<size_t>(d) * 4;
+    const size_t wbytes = static_cast<size_t>((d + 31) / 32) * 4;
+    bool vec = true;
+    for (int m = 0; m < M; ++m) {
+        if (grads[m] == nullptr) return SS_ERR_INVALID_ARG;
+        if (!aligned(grads[m], eb)) return SS_ERR_MISALIGNED;
+        vec = vec && aligned(grads[m], eb * 4);
+        if (momenta != nullptr) {
+            if (momenta[m] == nullptr) return SS_ERR_INVALID_ARG;
+            if (!aligned(momenta[m], 4)) return SS_ERR_MISALIGNED;
+            vec = vec && aligned(momenta[m], 16);
+            if (overlap(momenta[m], fbytes, grads[m], gbytes)) return SS_ERR_INVALID_ARG;
+            if (param != nullptr && overlap(momenta[m], fbytes, param, fbytes)) return SS_ERR_INVALID_ARG;
+            for (int k = 0; k < m; ++k)
+                if (overlap(momenta[m], fbytes, momenta[k], fbytes)) return SS_ERR_INVALID_ARG;
+        }
+        if (param != nullptr && overlap(grads[m], gbytes, param, fbytes)) return SS_ERR_INVALID_ARG;
+        if (words != nullptr && overlap(grads[m], gbytes, words, wbytes)) return SS_ERR_INVALID_ARG;
+    }
+    if (param != nullptr) {
+        if (!aligned(param, 4)) return SS_ERR_MISALIGNED;
+        vec = vec && aligned(param, 16);
+        if (words != nullptr && overlap(param, fbytes, words, wbytes)) return SS_ERR_INVALID_ARG;
+    }
+    if (words != nullptr && !aligned(words, 4)) return SS_ERR_MISALIGNED;
+
+    StepDesc s;
+    s.g = grads;
+    s.v = momenta;
+    s.M = M;
+    s.d = d;
+    s.beta = momenta != nullptr ? beta : 0.0f;
+    s.omb = 1.0f - s.beta;
+    s.lr = lr;
+    s.wd = weight_decay;
+    s.flip = flip_mask;
+    s.x = param;
+    s.words = words;
+    s.vec = vec;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    return cuda_status(dt == SS_F32 ? launch_step_f32(s, st) : launch_step_bf16(s, st));
+}
+
+int ss_sign_pack(const void* grad, ss_dtype dt, int64_t d, uint32_t* out_words, void* cuda_stream) {
+    if (grad == nullptr || (out_words == nullptr && d > 0)) return SS_ERR_INVALID_ARG;
+    const void* g[1] = {grad};
+    return step_common(g, dt, nullptr, 1, d, 0.0f, 0, nullptr, 0.0f, 0.0f, out_words, cuda_stream);
+}
+
+int ss_signum_update(const void* grad, ss_dtype dt, float* momentum, float beta, int64_t d,
+                     uint32_t* out_words, void* cuda_stream) {
+    if (grad == nullptr || momentum == nullptr || (out_words == nullptr && d > 0)) return SS_ERR_INVALID_ARG;
+    if (d > 0 && overlap(momentum, static_cast<size_t>(d) * 4, out_words, static_cast<size_t>((d + 31) / 32) * 4))
+        return SS_ERR_INVALID_ARG;
+    const void* g[1] = {grad};
+    float* v[1] = {momentum};
+    return step_common(g, dt, v, 1, d, beta, 0, nullptr, 0.0f, 0.0f, out_words, cuda_stream);
+}
+
+int ss_fused_step(const void* const* grads, ss_dtype dt, float* const* momenta, int M, int64_t d,
+                  float beta, uint64_t flip_mask, float* param, float lr, float weight_decay,
+                  uint32_t* vote_words_out, void* cuda_stream) {
+    if (param == nullptr) return SS_ERR_INVALID_ARG;
+    if (momenta != nullptr && vote_words_out != nullptr && d > 0 && M >= 1 && M <= SS_MAX_WORKERS) {
+        const size_t fbytes = static_cast<size_t>(d) * 4, wbytes = static_cast<size_t>((d + 31) / 32) * 4;
+        for (int m = 0; m < M; ++m)
+            if (momenta[m] != nullptr && overlap(momenta[m], fbytes, vote_words_out, wbytes)) return SS_ERR_INVALID_ARG;
+    }
+    return step_common(grads, dt, momenta, M, d, beta, flip_mask, param, lr, weight_decay,
+                       vote_words_out, cuda_stream);
+}
+
+int ss_majority_vote(const uint32_t* const* packed, int M, int64_t d, uint64_t flip_mask,
+                     uint32_t* vote_words, void* cuda_stream) {
+    if (packed == nullptr || M < 1 || M > SS_MAX_WORKERS || d < 0) return SS_ERR_INVALID_ARG;
+    if (!flip_ok(flip_mask, M)) return SS_ERR_INVALID_ARG;
+    if (d == 0) return SS_OK;
+    if (vote_words == nullptr) return SS_ERR_INVALID_ARG;
+    if (!aligned(vote_words, 4)) return SS_ERR_MISALIGNED;
+    const size_t wbytes = static_cast<size_t>((d + 31) / 32) * 4;
+    bool vec = aligned(vote_words, 16);
+    for (int m = 0; m < M; ++m) {
+        if (packed[m] == nullptr) return SS_ERR_INVALID_ARG;
+        if (!aligned(packed[m], 4)) return SS_ERR_MISALIGNED;
+        if (overlap(packed[m], wbytes, vote_words, wbytes)) return SS_ERR_INVALID_ARG;
+        vec = vec && aligned(packed[m], 16);
+    }
+    return cuda_status(launch_vote(packed, M, d, flip_mask, vote_words, vec,
+                                   static_cast<cudaStream_t>(cuda_stream)));
+}
+
+int ss_apply_vote(float* param, const uint32_t* vote_words, int64_t d, float lr, float weight_decay,
+                  void* cuda_stream) {
+    if (d < 0) return SS_ERR_INVALID_ARG;
+    if (d == 0) return SS_OK;
+    if (param == nullptr || vote_words == nullptr) return SS_ERR_INVALID_ARG;
+    if (!aligned(param, 4) || !aligned(vote_words, 4)) return SS_ERR_MISALIGNED;
+    if (overlap(param, static_cast<size_t>(d) * 4, vote_words, static_cast<size_t>((d + 31) / 32) * 4))
+        return SS_ERR_INVALID_ARG;
+    return cuda_status(launch_apply(param, vote_words, d, lr, weight_decay, aligned(param, 16),
+                                    static_cast<cudaStream_t>(cuda_stream)));
+}
+
+int ss_fused_step_host(const void* const* host_grads, ss_dtype dt, void* const* staging,
+                       float* const* momenta, int M, int64_t d, float beta, uint64_t flip_mask,
+                       float* param, float lr, float weight_decay, uint32_t* vote_words_dev,
+                       uint32_t* host_vote_out, void* cuda_stream) {
+    if (!dtype_ok(dt) || host_grads == nullptr || staging == nullptr || M < 1 || M > SS_MAX_WORKERS || d < 0)
+        return SS_ERR_INVALID_ARG;
+    if (d == 0) return SS_OK;
+    if (vote_words_dev == nullptr || param == nullptr) return SS_ERR_INVALID_ARG;
+    for (int m = 0; m < M; ++m)
+        if (host_grads[m] == nullptr || staging[m] == nullptr) return SS_ERR_INVALID_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    const size_t gbytes = static_cast<size_t>(d) * static_cast<size_t>(elem_bytes(dt));
+    for (int m = 0; m < M; ++m) {
+        cudaError_t e = cudaMemcpyAsync(staging[m], host_grads[m], gbytes, cudaMemcpyHostToDevice, st);
+        if (e != cudaSuccess) return cuda_status(e);
+    }
+    const int rc = step_common(reinterpret_cast<const void* const*>(staging), dt, momenta, M, d, beta,
+                               flip_mask, param, lr, weight_decay, vote_words_dev, cuda_stream);
+    if (rc != SS_OK) return rc;
+    if (host_vote_out != nullptr) {
+        cudaError_t e = cudaMemcpyAsync(host_vote_out, vote_words_dev,
+                                        static_cast<size_t>((d + 31) / 32) * 4, cudaMemcpyDeviceToHost, st);
+        if (e != cudaSuccess) return cuda_status(e);
+    }
+    return SS_OK;
+}
+
+#pragma GCC visibility pop
+}  // extern "C"

@@ -1,0 +1,130 @@
+// Shared device helpers: streaming loads/stores, the 1-bit sign, and the fp32 arithmetic of
+// Algorithm 1 written with explicitly rounded intrinsics so that no multiply-add is fused.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/signsgd.h"
+
+namespace ss {
+
+struct F32 {
+    static constexpr int kBytes = 4;
+    // four consecutive coordinates starting at coordinate 4 q
+    static __device__ __forceinline__ float4 load4(const void* base, int64_t q) {
+        return __ldcs(reinterpret_cast<const float4*>(base) + q);
+    }
+    static __device__ __forceinline__ float load1(const void* base, int64_t c) {
+        return __ldcs(reinterpret_cast<const float*>(base) + c);
+    }
+};
+
+struct BF16 {
+    static constexpr int kBytes = 2;
+    static __device__ __forceinline__ float4 load4(const void* base, int64_t q) {
+        const uint2 r = __ldcs(reinterpret_cast<const uint2*>(base) + q);
+        float4 f;
+        f.x = __uint_as_float(r.x << 16);
+        f.y = __uint_as_float(r.x & 0xFFFF0000u);
+        f.z = __uint_as_float(r.y << 16);
+        f.w = __uint_as_float(r.y & 0xFFFF0000u);
+        return f;
+    }
+    static __device__ __forceinline__ float load1(const void* base, int64_t c) {
+        const unsigned short h = __ldcs(reinterpret_cast<const unsigned short*>(base) + c);
+        return __uint_as_float(static_cast<uint32_t>(h) << 16);
+    }
+};
+
+// sign(z) as one bit: 1 iff z >= 0 by value (so +-0 -> 1, NaN -> 0).
+__device__ __forceinline__ uint32_t sign_bit(float z) { return z >= 0.0f ? 1u : 0u; }
+
+__device__ __forceinline__ uint32_t sign_nibble(const float4& s) {
+    return sign_bit(s.x) | (sign_bit(s.y) << 1) | (sign_bit(s.z) << 2) | (sign_bit(s.w) << 3);
+}
+
+// v <- (1 - beta) g + beta v: two rounded multiplies, one rounded add (Algorithm 1, momentum).
+__device__ __forceinline__ float momentum_rn(float omb, float g, float beta, float v) {
+    return __fadd_rn(__fmul_rn(omb, g), __fmul_rn(beta, v));
+}
+
+__device__ __forceinline__ float4 momentum_rn4(float omb, const float4& g, float beta,
+                                               const float4& v) {
+    float4 r;
+    r.x = momentum_rn(omb, g.x, beta, v.x);
+    r.y = momentum_rn(omb, g.y, beta, v.y);
+    r.z = momentum_rn(omb, g.z, beta, v.z);
+    r.w = momentum_rn(omb, g.w, beta, v.w);
+    return r;
+}
+
+// x <- x - lr (s + wd x), s = +1 if plus else -1 (Algorithm 1, parameter update).
+__device__ __forceinline__ float update_rn(float x, uint32_t plus, float lr, float wd,
+                                           bool has_wd) {
+    if (!has_wd) return __fsub_rn(x, plus ? lr : -lr);
+    const float s = plus ? 1.0f : -1.0f;
+    return __fsub_rn(x, __fmul_rn(lr, __fadd_rn(s, __fmul_rn(wd, x))));
+}
+
+__device__ __forceinline__ float4 update_rn4(const float4& x, uint32_t nib, float lr, float wd,
+                                             bool has_wd) {
+    float4 r;
+    r.x = update_rn(x.x, nib & 1u, lr, wd, has_wd);
+    r.y = update_rn(x.y, nib & 2u, lr, wd, has_wd);
+    r.z = update_rn(x.z, nib & 4u, lr, wd, has_wd);
+    r.w = update_rn(x.w, nib & 8u, lr, wd, has_wd);
+    return r;
+}
+
+// ---- host side --------------------------------------------------------------------------
+
+struct LaunchOptions {
+    int threads = 0;        // 0: kernel default
+    int blocks_per_sm = 0;  // 0: occupancy limit
+};
+LaunchOptions& launch_options();
+int device_sm_count(cudaError_t* err);
+
+// persistent grid: as many blocks as are resident at once, but no more than the work needs
+template <typename Kernel>
+inline cudaError_t persistent_grid(Kernel kernel, int threads, int64_t blocks_needed,
+                                   int* grid_out) {
+    cudaError_t err = cudaSuccess;
+    const int sms = device_sm_count(&err);
+    if (err != cudaSuccess) return err;
+    int per_sm = launch_options().blocks_per_sm;
+    if (per_sm <= 0) {
+        err = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, threads, 0);
+        if (err != cudaSuccess) return err;
+        if (per_sm < 1) per_sm = 1;
+    }
+    int64_t grid = static_cast<int64_t>(sms) * per_sm;
+    if (grid > blocks_needed) grid = blocks_needed;
+    if (grid < 1) grid = 1;
+    *grid_out = static_cast<int>(grid);
+    return cudaSuccess;
+}
+
+// ---- launch descriptors (filled by the C ABI after validation) ------------------------------
+
+struct StepDesc {
+    const void* const* g;   // M device pointers (host array)
+    float* const* v;        // M device pointers (host array) or null
+    int M;
+    int64_t d;
+    float beta, omb, lr, wd;
+    uint64_t flip;
+    float* x;               // null: no parameter update (pack only)
+    uint32_t* words;        // may be null when x != null
+    bool vec;               // all pointers sufficiently aligned for 128-bit access
+};
+
+cudaError_t launch_step_f32(const StepDesc& s, cudaStream_t st);
+cudaError_t launch_step_bf16(const StepDesc& s, cudaStream_t st);
+cudaError_t launch_vote(const uint32_t* const* packed, int M, int64_t d, uint64_t flip,
+                        uint32_t* vote, bool vec, cudaStream_t st);
+cudaError_t launch_apply(float* x, const uint32_t* vote, int64_t d, float lr, float wd, bool vec,
+                         cudaStream_t st);
+
+}  // namespace ss

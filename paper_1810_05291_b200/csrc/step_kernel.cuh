@@ -1,0 +1,270 @@
+// The streaming kernel behind ss_sign_pack, ss_signum_update and ss_fused_step: per coordinate,
+// Algorithm 1's momentum update, 1-bit sign, majority vote over the M workers and parameter
+// update, in one pass over memory.
+//
+// Vector form: a thread owns U quads (4 consecutive coordinates each). For every worker it
+// loads one 128-bit quad of the gradient (64-bit for bf16) and of the momentum, forms a 4-bit
+// sign nibble, and feeds the nibbles to a bit-sliced carry-save counter held in registers. The
+// vote nibble updates the thread's quad of x; eight neighbouring lanes OR their nibbles into one
+// canonical packed word. Loads are issued in batches of LB workers so that several 128-bit
+// requests per thread are in flight before the first is consumed.
+//
+// Ballot form: lane l of a warp owns coordinate 32 j + l of word j; __ballot_sync yields worker
+// m's canonical packed word directly and the counter runs on whole words, uniformly across the
+// warp. It needs only element alignment, handles the ragged last word, and is the fallback when
+// a pointer is not 16-byte aligned.
+#pragma once
+
+#include <type_traits>
+
+#include "bitslice.cuh"
+#include "common.cuh"
+
+namespace ss {
+
+template <int NP>
+struct StepArgs {
+    const void* g[NP];
+    float* v[NP];
+    float* x;
+    uint32_t* words;
+    int64_t d;
+    uint64_t flip;
+    float beta, omb, lr, wd;
+    int M;
+};
+
+template <int M_CT, bool MOM>
+struct StepShape {
+    static constexpr int NP = M_CT > 0 ? M_CT : SS_MAX_WORKERS;
+    static constexpr int P = M_CT > 0 ? bit_length(M_CT) : bit_length(SS_MAX_WORKERS);
+    static constexpr int IN_FLIGHT = MOM ? 4 : 8;  // worker quads loaded per batch (x2 with momentum)
+    static constexpr int LB = M_CT > 0 ? (M_CT < IN_FLIGHT ? M_CT : IN_FLIGHT) : 4;
+    static constexpr int U = (IN_FLIGHT / LB) > 0 ? (IN_FLIGHT / LB) : 1;
+};
+
+// One ragged or unaligned word: executed by a full warp, lane = bit position. M_CT = 0 loops
+// over the workers at run time (a.M of them, pointers indexed dynamically out of the NP slots).
+template <int M_CT, int NP, typename GT, bool MOM, bool APPLY>
+__device__ __forceinline__ void step_word_ballot(const StepArgs<NP>& a, int64_t j, int lane) {
+    constexpr int P = M_CT > 0 ? bit_length(M_CT) : bit_length(NP);
+    constexpr int LB = StepShape<M_CT, MOM>::LB;
+    const int M = M_CT > 0 ? M_CT : a.M;
+    const int64_t c = 32 * j + lane;
+    const bool valid = c < a.d;
+    const uint32_t vmask = __ballot_sync(0xFFFFFFFFu, valid);
+
+    BitCounter<P> cnt;
+    cnt.clear();
+    float xs = 0.0f;
+    if (APPLY && valid) xs = a.x[c];
+
+    auto batch = [&](int m0, auto nb_tag) {
+        constexpr int NB = decltype(nb_tag)::value;
+        float gs[NB], vs[NB];
+#pragma unroll
+        for (int k = 0; k < NB; ++k) {
+            const bool on = valid && (M_CT > 0 || m0 + k < M);
+            gs[k] = on ? GT::load1(a.g[m0 + k < NP ? m0 + k : 0], c) : -1.0f;
+            if (MOM) vs[k] = on ? __ldcs(a.v[m0 + k < NP ? m0 + k : 0] + c) : 0.0f;
+        }
+        uint32_t w[NB];
+#pragma unroll
+        for (int k = 0; k < NB; ++k) {
+            const bool live = (M_CT > 0 || m0 + k < M);
+            const bool on = valid && live;
+            float s = gs[k];
+            if (MOM) {
+                s = momentum_rn(a.omb, gs[k], a.beta, vs[k]);
+                if (on) __stcs(a.v[m0 + k < NP ? m0 + k : 0] + c, s);
+            }
+            const uint32_t word = __ballot_sync(0xFFFFFFFFu, on && s >= 0.0f);
+            const uint32_t fm = (0u - static_cast<uint32_t>((a.flip >> (m0 + k)) & 1ull)) & vmask;
+            w[k] = live ? (word ^ fm) : 0u;
+        }
+        cnt.template add_words<NB>(w);
+    };
+
+    if constexpr (M_CT > 0) {
+        constexpr int FULL = M_CT / LB, REM = M_CT % LB;
+#pragma unroll
+        for (int b = 0; b < FULL; ++b) batch(b * LB, std::integral_constant<int, LB>{});
+        if constexpr (REM > 0) batch(FULL * LB, std::integral_constant<int, REM>{});
+    } else {
+        for (int m0 = 0; m0 < M; m0 += LB) batch(m0, std::integral_constant<int, LB>{});
+    }
+
+    const uint32_t T = static_cast<uint32_t>(M + 1) >> 1;  // ceil(M/2): a tie votes +1
+    const uint32_t vote = cnt.at_least(T) & vmask;
+    if (APPLY && valid) a.x[c] = update_rn(xs, (vote >> lane) & 1u, a.lr, a.wd, a.wd != 0.0f);
+    if (lane == 0 && a.words != nullptr) a.words[j] = vote;
+}
+
+template <int M_CT, typename GT, bool MOM, bool APPLY>
+__global__ void __launch_bounds__(256)
+step_vec_kernel(const __grid_constant__ StepArgs<StepShape<M_CT, MOM>::NP> a) {
+    using S = StepShape<M_CT, MOM>;
+    constexpr int LB = S::LB, U = S::U;
+    const int M = M_CT > 0 ? M_CT : a.M;
+    const int lane = threadIdx.x & 31;
+    const int64_t n_quads = (a.d >> 5) << 3;  // quads lying in complete words
+    const int64_t tile = static_cast<int64_t>(blockDim.x) * U;
+    const uint32_t T = static_cast<uint32_t>(M + 1) >> 1;
+    const bool has_wd = a.wd != 0.0f;
+    const uint32_t group = 0xFFu << (lane & 24);  // the 8 lanes that share one packed word
+
+    for (int64_t base = static_cast<int64_t>(blockIdx.x) * tile; base < n_quads;
+         base += static_cast<int64_t>(gridDim.x) * tile) {
+        int64_t q[U];
+        bool ok[U];
+        float4 xq[U];
+        BitCounter<S::P> cnt[U];
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            q[u] = base + static_cast<int64_t>(u) * blockDim.x + threadIdx.x;
+            ok[u] = q[u] < n_quads;  // uniform over each 8-lane group: n_quads is a multiple of 8
+            cnt[u].clear();
+            if (APPLY && ok[u]) xq[u] = __ldcs(reinterpret_cast<const float4*>(a.x) + q[u]);
+        }
+
+        auto batch = [&](int m0, auto nb_tag) {
+            constexpr int NB = decltype(nb_tag)::value;
+            float4 gq[U][NB], vq[U][NB];
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+#pragma unroll
+                for (int k = 0; k < NB; ++k) {
+                    const bool on = ok[u] && (M_CT > 0 || m0 + k < M);
+                    const int mi = m0 + k < S::NP ? m0 + k : 0;
+                    gq[u][k] = on ? GT::load4(a.g[mi], q[u]) : make_float4(-1.f, -1.f, -1.f, -1.f);
+                    if (MOM)
+                        vq[u][k] = on ? __ldcs(reinterpret_cast<const float4*>(a.v[mi]) + q[u])
+                                      : make_float4(0.f, 0.f, 0.f, 0.f);
+                }
+            }
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                uint32_t nib[NB];
+#pragma unroll
+                for (int k = 0; k < NB; ++k) {
+                    const bool live = (M_CT > 0 || m0 + k < M);
+                    const int mi = m0 + k < S::NP ? m0 + k : 0;
+                    float4 s = gq[u][k];
+                    if (MOM) {
+                        s = momentum_rn4(a.omb, gq[u][k], a.beta, vq[u][k]);
+                        if (ok[u] && live) __stcs(reinterpret_cast<float4*>(a.v[mi]) + q[u], s);
+                    }
+                    // an inverting worker's nibble is complemented, branch-free
+                    const uint32_t fm = (0u - static_cast<uint32_t>((a.flip >> (m0 + k)) & 1ull)) & 0xFu;
+                    nib[k] = live ? (sign_nibble(s) ^ fm) : 0u;
+                }
+                cnt[u].template add_words<NB>(nib);
+            }
+        };
+
+        if constexpr (M_CT > 0) {
+            constexpr int FULL = M_CT / LB, REM = M_CT % LB;
+#pragma unroll
+            for (int b = 0; b < FULL; ++b) batch(b * LB, std::integral_constant<int, LB>{});
+            if constexpr (REM > 0) batch(FULL * LB, std::integral_constant<int, REM>{});
+        } else {
+            for (int m0 = 0; m0 < M; m0 += LB) batch(m0, std::integral_constant<int, LB>{});
+        }
+
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            if (ok[u]) {
+                const uint32_t vote = cnt[u].at_least(T) & 0xFu;
+                if (APPLY)
+                    __stcs(reinterpret_cast<float4*>(a.x) + q[u],
+                           update_rn4(xq[u], vote, a.lr, a.wd, has_wd));
+                if (a.words != nullptr) {
+                    const uint32_t w = __reduce_or_sync(group, vote << ((lane & 7) * 4));
+                    if ((lane & 7) == 0) a.words[q[u] >> 3] = w;
+                }
+            }
+        }
+    }
+
+    // the ragged last word (d not a multiple of 32): one warp, ballot form, run-time worker loop
+    if ((a.d & 31) != 0 && blockIdx.x == 0 && threadIdx.x < 32)
+        step_word_ballot<(M_CT == 1 ? 1 : 0), S::NP, GT, MOM, APPLY>(a, a.d >> 5, lane);
+}
+
+template <int M_CT, typename GT, bool MOM, bool APPLY>
+__global__ void __launch_bounds__(256)
+step_ballot_kernel(const __grid_constant__ StepArgs<StepShape<M_CT, MOM>::NP> a) {
+    const int lane = threadIdx.x & 31;
+    const int64_t W = (a.d + 31) >> 5;
+    const int64_t warps = (static_cast<int64_t>(gridDim.x) * blockDim.x) >> 5;
+    for (int64_t j = (static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x) >> 5; j < W;
+         j += warps)
+        step_word_ballot<M_CT, StepShape<M_CT, MOM>::NP, GT, MOM, APPLY>(a, j, lane);
+}
+
+template <int M_CT, typename GT, bool MOM, bool APPLY, bool VEC>
+cudaError_t launch_step_inst(const StepDesc& s, cudaStream_t st) {
+    using S = StepShape<M_CT, MOM>;
+    StepArgs<S::NP> a;
+    for (int m = 0; m < S::NP; ++m) {
+        a.g[m] = m < s.M ? s.g[m] : nullptr;
+        a.v[m] = (MOM && m < s.M) ? s.v[m] : nullptr;
+    }
+    a.x = s.x;
+    a.words = s.words;
+    a.d = s.d;
+    a.flip = s.flip;
+    a.beta = s.beta;
+    a.omb = s.omb;
+    a.lr = s.lr;
+    a.wd = s.wd;
+    a.M = s.M;
+    int threads = launch_options().threads > 0 ? launch_options().threads : 256;
+    if (threads > 256) threads = 256;
+    int grid = 1;
+    cudaError_t err;
+    if constexpr (VEC) {
+        auto kernel = step_vec_kernel<M_CT, GT, MOM, APPLY>;
+        const int64_t quads = (s.d >> 5) << 3;
+        const int64_t tile = static_cast<int64_t>(threads) * S::U;
+        err = persistent_grid(kernel, threads, (quads + tile - 1) / tile, &grid);
+        if (err != cudaSuccess) return err;
+        kernel<<<grid, threads, 0, st>>>(a);
+    } else {
+        auto kernel = step_ballot_kernel<M_CT, GT, MOM, APPLY>;
+        const int64_t W = (s.d + 31) >> 5;
+        const int64_t per_block = threads / 32;
+        err = persistent_grid(kernel, threads, (W + per_block - 1) / per_block, &grid);
+        if (err != cudaSuccess) return err;
+        kernel<<<grid, threads, 0, st>>>(a);
+    }
+    return cudaGetLastError();
+}
+
+// dispatch on (M, momentum, apply, alignment) for one gradient dtype. The vector form is
+// specialised for the worker counts of the paper's experiments and of the sweep (all 2^k - 1,
+// plus 16 for the even-M probe); any other M, and every unaligned call, takes the runtime-M form.
+template <typename GT>
+cudaError_t launch_step_dtype(const StepDesc& s, cudaStream_t st) {
+    const bool mom = s.v != nullptr;
+    const bool apply = s.x != nullptr;
+#define SS_STEP_PICK(MV, AP, VC)                                             \
+    (mom ? launch_step_inst<MV, GT, true, AP, VC>(s, st)                     \
+         : launch_step_inst<MV, GT, false, AP, VC>(s, st))
+    if (!apply)  // per-worker packing: M == 1 by construction
+        return s.vec ? SS_STEP_PICK(1, false, true) : SS_STEP_PICK(1, false, false);
+    if (!s.vec) return SS_STEP_PICK(0, true, false);
+    switch (s.M) {
+        case 1: return SS_STEP_PICK(1, true, true);
+        case 3: return SS_STEP_PICK(3, true, true);
+        case 7: return SS_STEP_PICK(7, true, true);
+        case 15: return SS_STEP_PICK(15, true, true);
+        case 16: return SS_STEP_PICK(16, true, true);
+        case 31: return SS_STEP_PICK(31, true, true);
+        case 63: return SS_STEP_PICK(63, true, true);
+        default: return SS_STEP_PICK(0, true, true);
+    }
+#undef SS_STEP_PICK
+}
+
+}  // namespace ss

@@ -1,0 +1,252 @@
+// ss_majority_vote and ss_apply_vote kernels: the server's and the workers' halves of
+// Algorithm 1 on already packed words (the unfused form a multi-GPU worker would use).
+#include <type_traits>
+
+#include "bitslice.cuh"
+#include "common.cuh"
+
+namespace ss {
+
+template <int NP>
+struct VoteArgs {
+    const uint32_t* p[NP];
+    uint32_t* out;
+    int64_t d;
+    uint64_t flip;
+    int M;
+};
+
+template <int M_CT>
+struct VoteShape {
+    static constexpr int NP = M_CT > 0 ? M_CT : SS_MAX_WORKERS;
+    static constexpr int P = M_CT > 0 ? bit_length(M_CT) : bit_length(SS_MAX_WORKERS);
+    static constexpr int LB = M_CT > 0 ? (M_CT < 8 ? M_CT : 8) : 4;
+};
+
+// mask of the valid bits of word j (only the last word can be ragged)
+__device__ __forceinline__ uint32_t valid_bits(int64_t j, int64_t d) {
+    const int64_t W = (d + 31) >> 5;
+    const int r = static_cast<int>(d & 31);
+    return (j == W - 1 && r != 0) ? ((1u << r) - 1u) : 0xFFFFFFFFu;
+}
+
+// one word per thread, 32-bit loads (tail words and the unaligned fallback)
+template <int M_CT>
+__device__ __forceinline__ void vote_one_word(const VoteArgs<VoteShape<M_CT>::NP>& a, int64_t j) {
+    using S = VoteShape<M_CT>;
+    constexpr int LB = S::LB;
+    const int M = M_CT > 0 ? M_CT : a.M;
+    BitCounter<S::P> cnt;
+    cnt.clear();
+    auto batch = [&](int m0, auto nb_tag) {
+        constexpr int NB = decltype(nb_tag)::value;
+        uint32_t w[NB];
+#pragma unroll
+        for (int k = 0; k < NB; ++k) {
+            const bool live = (M_CT > 0 || m0 + k < M);
+            const int mi = m0 + k < S::NP ? m0 + k : 0;
+            w[k] = live ? __ldcs(a.p[mi] + j) : 0u;
+        }
+#pragma unroll
+        for (int k = 0; k < NB; ++k) {
+            const bool live = (M_CT > 0 || m0 + k < M);
+            if (live && ((a.flip >> (m0 + k)) & 1ull)) w[k] = ~w[k];
+        }
+        cnt.template add_words<NB>(w);
+    };
+    if constexpr (M_CT > 0) {
+        constexpr int FULL = M_CT / LB, REM = M_CT % LB;
+#pragma unroll
+        for (int b = 0; b < FULL; ++b) batch(b * LB, std::integral_constant<int, LB>{});
+        if constexpr (REM > 0) batch(FULL * LB, std::integral_constant<int, REM>{});
+    } else {
+        for (int m0 = 0; m0 < M; m0 += LB) batch(m0, std::integral_constant<int, LB>{});
+    }
+    const uint32_t T = static_cast<uint32_t>(M + 1) >> 1;
+    a.out[j] = cnt.at_least(T) & valid_bits(j, a.d);
+}
+
+// four words per thread, 128-bit loads
+template <int M_CT>
+__global__ void __launch_bounds__(256)
+vote_vec_kernel(const __grid_constant__ VoteArgs<VoteShape<M_CT>::NP> a) {
+    using S = VoteShape<M_CT>;
+    constexpr int LB = S::LB;
+    const int M = M_CT > 0 ? M_CT : a.M;
+    const int64_t W = (a.d + 31) >> 5;
+    const int64_t n_groups = W >> 2;
+    const uint32_t T = static_cast<uint32_t>(M + 1) >> 1;
+    const int64_t stride = static_cast<int64_t>(gridDim.x) * blockDim.x;
+    for (int64_t i = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x; i < n_groups;
+         i += stride) {
+        BitCounter<S::P> cnt[4];
+#pragma unroll
+        for (int c = 0; c < 4; ++c) cnt[c].clear();
+        auto batch = [&](int m0, auto nb_tag) {
+            constexpr int NB = decltype(nb_tag)::value;
+            uint4 r[NB];
+#pragma unroll
+            for (int k = 0; k < NB; ++k) {
+                const bool live = (M_CT > 0 || m0 + k < M);
+                const int mi = m0 + k < S::NP ? m0 + k : 0;
+                r[k] = live ? __ldcs(reinterpret_cast<const uint4*>(a.p[mi]) + i)
+                            : make_uint4(0u, 0u, 0u, 0u);
+            }
+            uint32_t w[4][NB];
+#pragma unroll
+            for (int k = 0; k < NB; ++k) {
+                const bool live = (M_CT > 0 || m0 + k < M);
+                const uint32_t f = (live && ((a.flip >> (m0 + k)) & 1ull)) ? 0xFFFFFFFFu : 0u;
+                w[0][k] = r[k].x ^ f;
+                w[1][k] = r[k].y ^ f;
+                w[2][k] = r[k].z ^ f;
+                w[3][k] = r[k].w ^ f;
+            }
+#pragma unroll
+            for (int c = 0; c < 4; ++c) cnt[c].template add_words<NB>(w[c]);
+        };
+        if constexpr (M_CT > 0) {
+            constexpr int FULL = M_CT / LB, REM = M_CT % LB;
+#pragma unroll
+            for (int b = 0; b < FULL; ++b) batch(b * LB, std::integral_constant<int, LB>{});
+            if constexpr (REM > 0) batch(FULL * LB, std::integral_constant<int, REM>{});
+        } else {
+            for (int m0 = 0; m0 < M; m0 += LB) batch(m0, std::integral_constant<int, LB>{});
+        }
+        uint4 o;
+        o.x = cnt[0].at_least(T);
+        o.y = cnt[1].at_least(T);
+        o.z = cnt[2].at_least(T);
+        o.w = cnt[3].at_least(T) & valid_bits(4 * i + 3, a.d);
+        __stcs(reinterpret_cast<uint4*>(a.out) + i, o);
+    }
+    // up to three words that do not fill a group of four
+    const int64_t rest = W & 3;
+    if (blockIdx.x == 0 && threadIdx.x < rest) vote_one_word<M_CT>(a, (n_groups << 2) + threadIdx.x);
+}
+
+template <int M_CT>
+__global__ void __launch_bounds__(256)
+vote_word_kernel(const __grid_constant__ VoteArgs<VoteShape<M_CT>::NP> a) {
+    const int64_t W = (a.d + 31) >> 5;
+    const int64_t stride = static_cast<int64_t>(gridDim.x) * blockDim.x;
+    for (int64_t j = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x; j < W; j += stride)
+        vote_one_word<M_CT>(a, j);
+}
+
+template <int M_CT, bool VEC>
+cudaError_t launch_vote_inst(const uint32_t* const* packed, int M, int64_t d, uint64_t flip,
+                             uint32_t* vote, cudaStream_t st) {
+    using S = VoteShape<M_CT>;
+    VoteArgs<S::NP> a;
+    for (int m = 0; m < S::NP; ++m) a.p[m] = m < M ? packed[m] : nullptr;
+    a.out = vote;
+    a.d = d;
+    a.flip = flip;
+    a.M = M;
+    int threads = launch_options().threads > 0 ? launch_options().threads : 256;
+    if (threads > 256) threads = 256;
+    const int64_t W = (d + 31) >> 5;
+    int grid = 1;
+    cudaError_t err;
+    if constexpr (VEC) {
+        auto kernel = vote_vec_kernel<M_CT>;
+        err = persistent_grid(kernel, threads, ((W >> 2) + threads - 1) / threads, &grid);
+        if (err != cudaSuccess) return err;
+        kernel<<<grid, threads, 0, st>>>(a);
+    } else {
+        auto kernel = vote_word_kernel<M_CT>;
+        err = persistent_grid(kernel, threads, (W + threads - 1) / threads, &grid);
+        if (err != cudaSuccess) return err;
+        kernel<<<grid, threads, 0, st>>>(a);
+    }
+    return cudaGetLastError();
+}
+
+cudaError_t launch_vote(const uint32_t* const* packed, int M, int64_t d, uint64_t flip,
+                        uint32_t* vote, bool vec, cudaStream_t st) {
+    if (!vec) return launch_vote_inst<0, false>(packed, M, d, flip, vote, st);
+    switch (M) {
+        case 1: return launch_vote_inst<1, true>(packed, M, d, flip, vote, st);
+        case 3: return launch_vote_inst<3, true>(packed, M, d, flip, vote, st);
+        case 7: return launch_vote_inst<7, true>(packed, M, d, flip, vote, st);
+        case 15: return launch_vote_inst<15, true>(packed, M, d, flip, vote, st);
+        case 16: return launch_vote_inst<16, true>(packed, M, d, flip, vote, st);
+        case 31: return launch_vote_inst<31, true>(packed, M, d, flip, vote, st);
+        case 63: return launch_vote_inst<63, true>(packed, M, d, flip, vote, st);
+        default: return launch_vote_inst<0, true>(packed, M, d, flip, vote, st);
+    }
+}
+
+// ---- apply: x <- x - lr (sign(V) + wd x) from packed vote words ------------------------------
+
+struct ApplyArgs {
+    float* x;
+    const uint32_t* vote;
+    int64_t d;
+    float lr, wd;
+};
+
+__device__ __forceinline__ void apply_one(const ApplyArgs& a, int64_t c, bool has_wd) {
+    const uint32_t w = __ldg(a.vote + (c >> 5));
+    a.x[c] = update_rn(a.x[c], (w >> (c & 31)) & 1u, a.lr, a.wd, has_wd);
+}
+
+__global__ void __launch_bounds__(256) apply_vec_kernel(const __grid_constant__ ApplyArgs a) {
+    constexpr int U = 4;
+    const bool has_wd = a.wd != 0.0f;
+    const int64_t n_quads = a.d >> 2;
+    const int64_t tile = static_cast<int64_t>(blockDim.x) * U;
+    for (int64_t base = static_cast<int64_t>(blockIdx.x) * tile; base < n_quads;
+         base += static_cast<int64_t>(gridDim.x) * tile) {
+        float4 xq[U];
+        uint32_t w[U];
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const int64_t q = base + static_cast<int64_t>(u) * blockDim.x + threadIdx.x;
+            if (q < n_quads) {
+                xq[u] = __ldcs(reinterpret_cast<const float4*>(a.x) + q);
+                w[u] = __ldg(a.vote + (q >> 3));
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const int64_t q = base + static_cast<int64_t>(u) * blockDim.x + threadIdx.x;
+            if (q < n_quads) {
+                const uint32_t nib = (w[u] >> ((q & 7) * 4)) & 0xFu;
+                __stcs(reinterpret_cast<float4*>(a.x) + q, update_rn4(xq[u], nib, a.lr, a.wd, has_wd));
+            }
+        }
+    }
+    const int64_t rest = a.d & 3;
+    if (blockIdx.x == 0 && threadIdx.x < rest) apply_one(a, (n_quads << 2) + threadIdx.x, has_wd);
+}
+
+__global__ void __launch_bounds__(256) apply_scalar_kernel(const __grid_constant__ ApplyArgs a) {
+    const bool has_wd = a.wd != 0.0f;
+    const int64_t stride = static_cast<int64_t>(gridDim.x) * blockDim.x;
+    for (int64_t c = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x; c < a.d; c += stride)
+        apply_one(a, c, has_wd);
+}
+
+cudaError_t launch_apply(float* x, const uint32_t* vote, int64_t d, float lr, float wd, bool vec,
+                         cudaStream_t st) {
+    ApplyArgs a{x, vote, d, lr, wd};
+    int threads = launch_options().threads > 0 ? launch_options().threads : 256;
+    if (threads > 256) threads = 256;
+    int grid = 1;
+    cudaError_t err;
+    if (vec) {
+        const int64_t tile = static_cast<int64_t>(threads) * 4;
+        err = persistent_grid(apply_vec_kernel, threads, ((d >> 2) + tile - 1) / tile, &grid);
+        if (err != cudaSuccess) return err;
+        apply_vec_kernel<<<grid, threads, 0, st>>>(a);
+    } else {
+        err = persistent_grid(apply_scalar_kernel, threads, (d + threads - 1) / threads, &grid);
+        if (err != cudaSuccess) return err;
+        apply_scalar_kernel<<<grid, threads, 0, st>>>(a);
+    }
+    return cudaGetLastError();
+}
+
+}  // namespace ss
