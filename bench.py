@@ -1,0 +1,395 @@
+#!/usr/bin/env python
+"""Benchmark of the fused Signum step (momentum -> sign -> majority vote -> update, one kernel).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload cfg3] [--impl ours|reference]
+
+A step is one call of ss_fused_step over one batch of synthetic gradients: M = 15 workers,
+d = 25,557,032 (ResNet-50-sized) fp32, per-worker momentum, beta = 0.9, lr = 1e-4. Under
+torchrun every rank runs the same workload on its own GPU (the path shards by coordinate and
+needs no collective), timing is the maximum over ranks, and rank 0 prints one JSON line.
+"""
+
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "fused pack+vote+apply params/s"
+UNIT = "params/s"
+FALLBACK_HBM_GBS = 6650.0
+NOMINAL_HBM_GBS = 8000.0
+
+
+def make_case(name: str, d_override=None):
+    from paper_1810_05291_b200 import inputs
+    if name == "cfg1":
+        c = inputs.cfg1()
+    elif name == "cfg2":
+        c = inputs.cfg2()
+    elif name == "cfg3":
+        c = inputs.cfg3()
+    elif name == "cfg4":
+        c = inputs.cfg4()
+    elif name == "cfg4tie":
+        c = inputs.cfg4(tie_probe=True)
+    elif name.startswith("sweep:"):          # sweep:<d>:<M>[:mom]
+        parts = name.split(":")
+        c = inputs.cfg5(int(parts[1]), int(parts[2]), momentum=len(parts) > 3)
+    else:
+        raise SystemExit("unknown workload %r" % name)
+    if d_override:
+        c.d = int(d_override)
+    return c
+
+
+def algorithmic_bytes(case) -> int:
+    """Bytes one fused step must move: per coordinate, M gradients read, (with momentum) M
+    momenta read and written, x read and written."""
+    import torch
+    gb = 4 if case.dtype == torch.float32 else 2
+    per = case.M * gb + 8
+    if case.beta is not None:
+        per += case.M * 8
+    return per * case.d
+
+
+def measured_peak():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured (MEASURED_PEAKS.json hbm_gbs, torch copy read+write)"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback (6.65 TB/s, earlier measurement on this pool)"
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons of one GPU with nvidia-smi while the timed region runs."""
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+              "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.proc = None
+        self.lines = []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.FIELDS,
+                 "--format=csv,noheader,nounits", "-lms", "100"],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append((time.time(), line.strip()))
+
+    def stop(self, t0: float, t1: float) -> dict:
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        rows = [l for (t, l) in self.lines if t0 <= t <= t1 + 0.2] or [l for (_, l) in self.lines]
+        sm, smax, power, reasons = [], [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in rows:
+            p = [x.strip() for x in r.split(",")]
+            if len(p) < 8:
+                continue
+            try:
+                sm.append(float(p[0]))
+                smax.append(float(p[1]))
+                power.append(float(p[2]))
+            except ValueError:
+                continue
+            for name, val in zip(names, p[4:8]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": statistics.median(sm) if sm else None,
+                "sm_max_mhz": max(smax) if smax else None,
+                "power_w_max": max(power) if power else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def time_oracle(case, steps: int, warmup: int, threads: int, budget_s: float = 12.0):
+    """Times the CPU oracle, as it stands, on a bounded sample of the workload: the first
+    d_s coordinates of all M workers (every coordinate is independent), d_s chosen so that the
+    run stays near budget_s seconds. Returns (params_per_s, d_s, threads_used, seconds_per_step)."""
+    import numpy as np
+    import torch
+
+    import oracle
+    from paper_1810_05291_b200 import inputs
+
+    oracle.set_threads(threads)
+    used = oracle.get_threads()
+    probe_d = min(case.d, 1 << 21)
+
+    def host_inputs(d_s):
+        sub = make_case_like(case, d_s)
+        grads = [to_host(g) for g in inputs.gradients(sub, "cpu", 0)]
+        x = inputs.initial_params(sub, "cpu").numpy().copy()
+        moms = [np.zeros(d_s, dtype=np.float32) for _ in range(sub.M)] if sub.beta is not None else None
+        return sub, grads, moms, x
+
+    def to_host(t):
+        if t.dtype == torch.bfloat16:
+            return t.view(torch.int16).numpy().view(np.uint16).copy()
+        return t.numpy().copy()
+
+    def run(sub, grads, moms, x, n):
+        t0 = time.perf_counter()
+        for _ in range(n):
+            oracle.fused_step(grads, moms, x, sub.beta if sub.beta is not None else 0.0, sub.lr,
+                              sub.weight_decay, sub.flip_mask)
+        return (time.perf_counter() - t0) / n
+
+    sub, grads, moms, x = host_inputs(probe_d)
+    run(sub, grads, moms, x, 1)
+    per_coord = run(sub, grads, moms, x, 2) / probe_d
+    total_steps = max(1, steps + warmup)
+    d_s = int(min(case.d, max(1 << 16, budget_s / (per_coord * total_steps))))
+    if d_s < case.d:
+        d_s = max(32, d_s - d_s % 32)
+    if d_s != probe_d:
+        sub, grads, moms, x = host_inputs(d_s)
+    run(sub, grads, moms, x, max(1, warmup))
+    sec = run(sub, grads, moms, x, max(1, steps))
+    oracle.set_threads(1)
+    return d_s / sec, d_s, used, sec
+
+
+def make_case_like(case, d):
+    import copy
+    c = copy.copy(case)
+    c.d = int(d)
+    return c
+
+
+def reference_arm(args) -> None:
+    """The reference arm of this benchmark is the CPU oracle, timed as it stands on the host cores."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import oracle
+    case = make_case(args.workload, args.d)
+    cores = oracle.max_threads()
+    value, d_s, used, sec = time_oracle(case, args.steps, args.warmup, cores)
+    sample = "first %d of %d coordinates, all %d workers, per step" % (d_s, case.d, case.M)
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": sec * 1e3 * case.d / d_s,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": dtype_name(case), "data": "synthetic",
+        "config": config_of(case, "host memory; CPU oracle"),
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": used, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+def dtype_name(case) -> str:
+    import torch
+    return "f32" if case.dtype == torch.float32 else "bf16 gradients, f32 state"
+
+
+def config_of(case, residency: str) -> dict:
+    return {"workload": case.name, "M": case.M, "d": case.d, "beta": case.beta, "lr": case.lr,
+            "weight_decay": case.weight_decay, "flip_mask": case.flip_mask,
+            "entry_point": "ss_fused_step", "l2": residency}
+
+
+def main() -> None:
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="cfg3")
+    ap.add_argument("--d", type=int, default=None, help="override the coordinate count (tests, profiling)")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--profile", action="store_true",
+                    help="for runs under a profiler: no clock sampling, no end-to-end and CPU legs")
+    ap.add_argument("--threads", type=int, default=0, help="launch-shape override: block size")
+    ap.add_argument("--blocks-per-sm", type=int, default=0, help="launch-shape override")
+    args = ap.parse_args()
+    if args.warmup < 3:
+        args.warmup = 3
+    if args.profile:
+        args.no_e2e = args.no_cpu_baseline = True
+
+    if args.impl == "reference":
+        reference_arm(args)
+        return
+
+    import torch
+    import torch.distributed as dist
+
+    from paper_1810_05291_b200 import binding as B
+    from paper_1810_05291_b200 import inputs
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the library has no CPU path")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        dist.init_process_group("nccl", device_id=dev)
+
+    B.lib()  # fail here, loudly, if the CUDA library is missing
+    if args.threads:
+        B.ss_set_launch_option("threads", args.threads)
+    if args.blocks_per_sm:
+        B.ss_set_launch_option("blocks_per_sm", args.blocks_per_sm)
+
+    case = make_case(args.workload, args.d)
+    case.cfg = case.cfg * 100 + rank  # every rank holds its own shard of coordinates: distinct data
+    grads = inputs.gradients(case, dev, 0)
+    x = inputs.initial_params(case, dev)
+    moms = inputs.zero_momenta(case, dev)
+    vote = torch.zeros(B.ss_packed_words(case.d), dtype=torch.int32, device=dev)
+    beta = case.beta if case.beta is not None else 0.0
+    stream = torch.cuda.current_stream()
+
+    def step():
+        B.ss_fused_step(grads, moms, x, beta, case.lr, case.weight_decay, case.flip_mask, vote, stream)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(args.warmup):
+        step()
+    barrier()
+    sampler = ClockSampler(local_rank if "CUDA_VISIBLE_DEVICES" not in os.environ
+                           else int(os.environ["CUDA_VISIBLE_DEVICES"].split(",")[local_rank]))
+    if not args.profile:
+        sampler.start()
+        time.sleep(0.3)
+        # a short spell of the same kernel so that clock samples are taken under load
+        for _ in range(args.warmup):
+            step()
+        barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t0 = time.time()
+    e0.record(stream)
+    for _ in range(args.steps):
+        step()
+    e1.record(stream)
+    barrier()
+    t1 = time.time()
+    ms_total = e0.elapsed_time(e1)
+    # keep the GPU busy a little longer if the timed region was too short for nvidia-smi to see
+    if t1 - t0 < 0.5 and not args.profile:
+        t_extra = time.time()
+        while time.time() - t_extra < 0.6:
+            for _ in range(20):
+                step()
+            torch.cuda.synchronize()
+        t1 = time.time()
+    clocks = sampler.stop(t0, t1) if not args.profile else {"sm_mhz": None, "reasons": ["not sampled (--profile)"]}
+
+    if world > 1:
+        t = torch.tensor([ms_total], device=dev, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms_total = float(t.item())
+    ms_step = ms_total / args.steps
+    value = world * case.d / (ms_step * 1e-3)
+
+    # ---- end to end: gradients start in pinned host memory, packed vote returns to the host ----
+    e2e = None
+    if not args.no_e2e:
+        host = [g.cpu().pin_memory() for g in grads]
+        hv = torch.zeros(vote.numel(), dtype=torch.int32).pin_memory()
+        n_e2e = max(3, min(args.steps, 10))
+
+        def step_host():
+            B.ss_fused_step_host(host, grads, moms, x, beta, case.lr, case.weight_decay,
+                                 case.flip_mask, vote, hv, stream)
+
+        for _ in range(2):
+            step_host()
+        barrier()
+        h0, h1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        h0.record(stream)
+        for _ in range(n_e2e):
+            step_host()
+        h1.record(stream)
+        barrier()
+        ms_e2e = h0.elapsed_time(h1)
+        if world > 1:
+            t = torch.tensor([ms_e2e], device=dev, dtype=torch.float64)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            ms_e2e = float(t.item())
+        e2e = {"value": world * case.d / (ms_e2e / n_e2e * 1e-3), "unit": UNIT,
+               "h2d_bytes_per_step": sum(h.numel() * h.element_size() for h in host),
+               "d2h_bytes_per_step": hv.numel() * 4, "steps": n_e2e,
+               "ms_per_step": ms_e2e / n_e2e, "entry_point": "ss_fused_step_host"}
+        del host
+
+    if rank == 0:
+        abytes = algorithmic_bytes(case)
+        peak, peak_src = measured_peak()
+        achieved = abytes / (ms_step * 1e-3) / 1e9
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": dtype_name(case), "data": "synthetic",
+            "config": config_of(case, "inputs %.2f GB per step, far larger than the 126 MB L2; no flush"
+                                % (abytes / 1e9)),
+            "hbm_gbs": achieved, "pct_of_nominal_8tbs": 100.0 * achieved / NOMINAL_HBM_GBS,
+            "gradient_elements_per_s": value * case.M,
+            "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
+                         "frac": achieved / peak, "traffic": None, "peak_source": peak_src,
+                         "kernel": "step_vec_kernel<M=%d,%s,momentum=%s,apply>" % (
+                             case.M, "f32" if case.dtype == torch.float32 else "bf16",
+                             "yes" if case.beta is not None else "no"),
+                         "algorithmic_bytes_per_launch": abytes,
+                         "launch_ms": ms_step},
+            "gpu_launches": args.steps,
+            "clocks": clocks,
+        }
+        if e2e is not None:
+            line["e2e"] = e2e
+        if world == 1 and not args.no_cpu_baseline:
+            import oracle
+            cores = oracle.max_threads()
+            v_all, d_s, used, _ = time_oracle(case, 3, 1, cores, budget_s=8.0)
+            v_one, d_1, _, _ = time_oracle(case, 2, 1, 1, budget_s=8.0)
+            line["cpu_baseline"] = {
+                "value": v_all, "unit": UNIT, "cores": used, "kind": "oracle",
+                "sample": "first %d of %d coordinates, all %d workers, 3 timed steps" % (d_s, case.d, case.M),
+                "value_1_thread": v_one,
+                "sample_1_thread": "first %d coordinates, 2 timed steps" % d_1}
+        print(json.dumps(line), flush=True)
+
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -89,10 +89,10 @@ int ss_set_launch_option(const char* key, int value) {
 static int step_common(const void* const* grads, ss_dtype dt, float* const* momenta, int M,
                        int64_t d, float beta, uint64_t flip_mask, float* param, float lr,
                        float weight_decay, uint32_t* words, void* cuda_stream) {
-    if (!dtype_ok(dt) || grads == nullptr || M < 1 || M > SS_MAX_WORKERS || d < 0) return SS_ERR_INVALID_ARG;
+    if (!dtype_ok(dt) || M < 1 || M > SS_MAX_WORKERS || d < 0) return SS_ERR_INVALID_ARG;
     if (!flip_ok(flip_mask, M)) return SS_ERR_INVALID_ARG;
     if (d == 0) return SS_OK;
-    if (param == nullptr && words == nullptr) return SS_ERR_INVALID_ARG;
+    if (grads == nullptr || (param == nullptr && words == nullptr)) return SS_ERR_INVALID_ARG;
     const size_t eb = static_cast<size_t>(elem_bytes(dt));
     const size_t gbytes = static_cast<size_t>(d) * eb, fbytes = static_cast<size_t>(d) * 4;
     const size_t wbytes = static_cast<size_t>((d + 31) / 32) * 4;
@@ -138,14 +138,14 @@ static int step_common(const void* const* grads, ss_dtype dt, float* const* mome
 }
 
 int ss_sign_pack(const void* grad, ss_dtype dt, int64_t d, uint32_t* out_words, void* cuda_stream) {
-    if (grad == nullptr || (out_words == nullptr && d > 0)) return SS_ERR_INVALID_ARG;
+    if (d > 0 && (grad == nullptr || out_words == nullptr)) return SS_ERR_INVALID_ARG;
     const void* g[1] = {grad};
     return step_common(g, dt, nullptr, 1, d, 0.0f, 0, nullptr, 0.0f, 0.0f, out_words, cuda_stream);
 }
 
 int ss_signum_update(const void* grad, ss_dtype dt, float* momentum, float beta, int64_t d,
                      uint32_t* out_words, void* cuda_stream) {
-    if (grad == nullptr || momentum == nullptr || (out_words == nullptr && d > 0)) return SS_ERR_INVALID_ARG;
+    if (d > 0 && (grad == nullptr || momentum == nullptr || out_words == nullptr)) return SS_ERR_INVALID_ARG;
     if (d > 0 && overlap(momentum, static_cast<size_t>(d) * 4, out_words, static_cast<size_t>((d + 31) / 32) * 4))
         return SS_ERR_INVALID_ARG;
     const void* g[1] = {grad};
@@ -156,7 +156,7 @@ int ss_signum_update(const void* grad, ss_dtype dt, float* momentum, float beta,
 int ss_fused_step(const void* const* grads, ss_dtype dt, float* const* momenta, int M, int64_t d,
                   float beta, uint64_t flip_mask, float* param, float lr, float weight_decay,
                   uint32_t* vote_words_out, void* cuda_stream) {
-    if (param == nullptr) return SS_ERR_INVALID_ARG;
+    if (d > 0 && param == nullptr) return SS_ERR_INVALID_ARG;
     if (momenta != nullptr && vote_words_out != nullptr && d > 0 && M >= 1 && M <= SS_MAX_WORKERS) {
         const size_t fbytes = static_cast<size_t>(d) * 4, wbytes = static_cast<size_t>((d + 31) / 32) * 4;
         for (int m = 0; m < M; ++m)
@@ -201,10 +201,11 @@ int ss_fused_step_host(const void* const* host_grads, ss_dtype dt, void* const* 
                        float* const* momenta, int M, int64_t d, float beta, uint64_t flip_mask,
                        float* param, float lr, float weight_decay, uint32_t* vote_words_dev,
                        uint32_t* host_vote_out, void* cuda_stream) {
-    if (!dtype_ok(dt) || host_grads == nullptr || staging == nullptr || M < 1 || M > SS_MAX_WORKERS || d < 0)
+    if (!dtype_ok(dt) || M < 1 || M > SS_MAX_WORKERS || d < 0 || !flip_ok(flip_mask, M))
         return SS_ERR_INVALID_ARG;
     if (d == 0) return SS_OK;
-    if (vote_words_dev == nullptr || param == nullptr) return SS_ERR_INVALID_ARG;
+    if (host_grads == nullptr || staging == nullptr || vote_words_dev == nullptr || param == nullptr)
+        return SS_ERR_INVALID_ARG;
     for (int m = 0; m < M; ++m)
         if (host_grads[m] == nullptr || staging[m] == nullptr) return SS_ERR_INVALID_ARG;
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);

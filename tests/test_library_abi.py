@@ -61,6 +61,7 @@ def test_argument_errors_are_reported_before_any_cuda_call(L):
     null_arr = (ctypes.c_void_p * 1)(None)
     # null pointers
     assert L.ss_sign_pack(None, 0, 10, fake, None) == B.SS_ERR_INVALID_ARG
+    assert L.ss_fused_step(None, 0, None, 1, 10, 0.0, 0, fake, 0.1, 0.0, None, None) == B.SS_ERR_INVALID_ARG
     assert L.ss_sign_pack(fake, 0, 10, None, None) == B.SS_ERR_INVALID_ARG
     assert L.ss_fused_step(arr1, 0, None, 1, 10, 0.0, 0, None, 0.1, 0.0, None, None) == B.SS_ERR_INVALID_ARG
     assert L.ss_fused_step(null_arr, 0, None, 1, 10, 0.0, 0, fake, 0.1, 0.0, None, None) == B.SS_ERR_INVALID_ARG
@@ -83,6 +84,9 @@ def test_argument_errors_are_reported_before_any_cuda_call(L):
     assert L.ss_apply_vote(fake, fake, 10, 0.1, 0.0, None) == B.SS_ERR_INVALID_ARG
     # d == 0 is a no-op
     assert L.ss_sign_pack(fake, 0, 0, None, None) == B.SS_OK
+    assert L.ss_sign_pack(None, 0, 0, None, None) == B.SS_OK
+    assert L.ss_fused_step(None, 0, None, 1, 0, 0.0, 0, None, 0.1, 0.0, None, None) == B.SS_OK
+    assert L.ss_fused_step(None, 0, None, 0, 0, 0.0, 0, None, 0.1, 0.0, None, None) == B.SS_ERR_INVALID_ARG
     assert L.ss_apply_vote(None, None, 0, 0.1, 0.0, None) == B.SS_OK
     assert L.ss_majority_vote(arr1, 1, 0, 0, None, None) == B.SS_OK
 

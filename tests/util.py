@@ -51,7 +51,12 @@ def assert_f32_close(got: torch.Tensor, want: np.ndarray, what: str = "fp32 stat
 
 
 def count_bit_mismatch(got: torch.Tensor, want: np.ndarray) -> int:
-    return int(np.count_nonzero(to_np(got).view(np.uint32) != want.view(np.uint32)))
+    """Elements whose fp32 bit patterns differ. A NaN on both sides counts as equal: the NaN
+    payload is the one thing IEEE 754 leaves to the implementation (x86 keeps the operand's
+    payload, the GPU returns the canonical NaN)."""
+    g = to_np(got)
+    both_nan = np.isnan(g) & np.isnan(want)
+    return int(np.count_nonzero((g.view(np.uint32) != want.view(np.uint32)) & ~both_nan))
 
 
 class GuardedWords:
