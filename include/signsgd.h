@@ -144,7 +144,8 @@ int ss_fused_step_host(const void* const* host_grads, ss_dtype dt, void* const* 
 /*
  * Launch-shape override for benchmarking sweeps (process-wide; not part of the method).
  *   key: "threads" (block size, multiple of 32 in [64, 1024], 0 = default) or
- *        "blocks_per_sm" (persistent blocks per SM, 0 = as many as fit).
+ *        "blocks_per_sm" (0 = one block per tile, the default; n > 0 = a persistent grid of
+        n blocks per SM that strides over the tiles; at most 4096).
  * Returns SS_ERR_INVALID_ARG for an unknown key or a value out of range.
  */
 int ss_set_launch_option(const char* key, int value);

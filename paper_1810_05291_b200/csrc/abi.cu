@@ -79,7 +79,7 @@ int ss_set_launch_option(const char* key, int value) {
         return SS_OK;
     }
     if (std::strcmp(key, "blocks_per_sm") == 0) {
-        if (value < 0 || value > 32) return SS_ERR_INVALID_ARG;
+        if (value < 0 || value > 4096) return SS_ERR_INVALID_ARG;
         launch_options().blocks_per_sm = value;
         return SS_OK;
     }

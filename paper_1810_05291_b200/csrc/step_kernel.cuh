@@ -26,6 +26,7 @@ template <int NP>
 struct StepArgs {
     const void* g[NP];
     float* v[NP];
+    uint32_t fnib[NP];  // 0xF for an inverting worker, else 0: XORed into its sign nibble
     float* x;
     uint32_t* words;
     int64_t d;
@@ -34,11 +35,19 @@ struct StepArgs {
     int M;
 };
 
+// Worker quads a thread requests per load batch (twice as many 128-bit loads with momentum).
+#ifndef SS_BATCH_MOMENTUM
+#define SS_BATCH_MOMENTUM 4
+#endif
+#ifndef SS_BATCH_PLAIN
+#define SS_BATCH_PLAIN 8
+#endif
+
 template <int M_CT, bool MOM>
 struct StepShape {
     static constexpr int NP = M_CT > 0 ? M_CT : SS_MAX_WORKERS;
     static constexpr int P = M_CT > 0 ? bit_length(M_CT) : bit_length(SS_MAX_WORKERS);
-    static constexpr int IN_FLIGHT = MOM ? 4 : 8;  // worker quads loaded per batch (x2 with momentum)
+    static constexpr int IN_FLIGHT = MOM ? SS_BATCH_MOMENTUM : SS_BATCH_PLAIN;
     static constexpr int LB = M_CT > 0 ? (M_CT < IN_FLIGHT ? M_CT : IN_FLIGHT) : 4;
     static constexpr int U = (IN_FLIGHT / LB) > 0 ? (IN_FLIGHT / LB) : 1;
 };
@@ -79,7 +88,7 @@ __device__ __forceinline__ void step_word_ballot(const StepArgs<NP>& a, int64_t 
                 if (on) __stcs(a.v[m0 + k < NP ? m0 + k : 0] + c, s);
             }
             const uint32_t word = __ballot_sync(0xFFFFFFFFu, on && s >= 0.0f);
-            const uint32_t fm = (0u - static_cast<uint32_t>((a.flip >> (m0 + k)) & 1ull)) & vmask;
+            const uint32_t fm = (0u - (a.fnib[m0 + k < NP ? m0 + k : 0] & 1u)) & vmask;
             w[k] = live ? (word ^ fm) : 0u;
         }
         cnt.template add_words<NB>(w);
@@ -154,9 +163,8 @@ step_vec_kernel(const __grid_constant__ StepArgs<StepShape<M_CT, MOM>::NP> a) {
                         s = momentum_rn4(a.omb, gq[u][k], a.beta, vq[u][k]);
                         if (ok[u] && live) __stcs(reinterpret_cast<float4*>(a.v[mi]) + q[u], s);
                     }
-                    // an inverting worker's nibble is complemented, branch-free
-                    const uint32_t fm = (0u - static_cast<uint32_t>((a.flip >> (m0 + k)) & 1ull)) & 0xFu;
-                    nib[k] = live ? (sign_nibble(s) ^ fm) : 0u;
+                    // an inverting worker's nibble is complemented (mask read from the parameters)
+                    nib[k] = live ? (sign_nibble(s) ^ a.fnib[mi]) : 0u;
                 }
                 cnt[u].template add_words<NB>(nib);
             }
@@ -209,6 +217,7 @@ cudaError_t launch_step_inst(const StepDesc& s, cudaStream_t st) {
     for (int m = 0; m < S::NP; ++m) {
         a.g[m] = m < s.M ? s.g[m] : nullptr;
         a.v[m] = (MOM && m < s.M) ? s.v[m] : nullptr;
+        a.fnib[m] = (m < s.M && ((s.flip >> m) & 1ull)) ? 0xFu : 0u;
     }
     a.x = s.x;
     a.words = s.words;
@@ -227,14 +236,14 @@ cudaError_t launch_step_inst(const StepDesc& s, cudaStream_t st) {
         auto kernel = step_vec_kernel<M_CT, GT, MOM, APPLY>;
         const int64_t quads = (s.d >> 5) << 3;
         const int64_t tile = static_cast<int64_t>(threads) * S::U;
-        err = persistent_grid(kernel, threads, (quads + tile - 1) / tile, &grid);
+        err = pick_grid(kernel, threads, (quads + tile - 1) / tile, &grid);
         if (err != cudaSuccess) return err;
         kernel<<<grid, threads, 0, st>>>(a);
     } else {
         auto kernel = step_ballot_kernel<M_CT, GT, MOM, APPLY>;
         const int64_t W = (s.d + 31) >> 5;
         const int64_t per_block = threads / 32;
-        err = persistent_grid(kernel, threads, (W + per_block - 1) / per_block, &grid);
+        err = pick_grid(kernel, threads, (W + per_block - 1) / per_block, &grid);
         if (err != cudaSuccess) return err;
         kernel<<<grid, threads, 0, st>>>(a);
     }

@@ -151,12 +151,12 @@ cudaError_t launch_vote_inst(const uint32_t* const* packed, int M, int64_t d, ui
     cudaError_t err;
     if constexpr (VEC) {
         auto kernel = vote_vec_kernel<M_CT>;
-        err = persistent_grid(kernel, threads, ((W >> 2) + threads - 1) / threads, &grid);
+        err = pick_grid(kernel, threads, ((W >> 2) + threads - 1) / threads, &grid);
         if (err != cudaSuccess) return err;
         kernel<<<grid, threads, 0, st>>>(a);
     } else {
         auto kernel = vote_word_kernel<M_CT>;
-        err = persistent_grid(kernel, threads, (W + threads - 1) / threads, &grid);
+        err = pick_grid(kernel, threads, (W + threads - 1) / threads, &grid);
         if (err != cudaSuccess) return err;
         kernel<<<grid, threads, 0, st>>>(a);
     }
@@ -238,11 +238,11 @@ cudaError_t launch_apply(float* x, const uint32_t* vote, int64_t d, float lr, fl
     cudaError_t err;
     if (vec) {
         const int64_t tile = static_cast<int64_t>(threads) * 4;
-        err = persistent_grid(apply_vec_kernel, threads, ((d >> 2) + tile - 1) / tile, &grid);
+        err = pick_grid(apply_vec_kernel, threads, ((d >> 2) + tile - 1) / tile, &grid);
         if (err != cudaSuccess) return err;
         apply_vec_kernel<<<grid, threads, 0, st>>>(a);
     } else {
-        err = persistent_grid(apply_scalar_kernel, threads, (d + threads - 1) / threads, &grid);
+        err = pick_grid(apply_scalar_kernel, threads, (d + threads - 1) / threads, &grid);
         if (err != cudaSuccess) return err;
         apply_scalar_kernel<<<grid, threads, 0, st>>>(a);
     }
