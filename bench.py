@@ -246,7 +246,7 @@ def main() -> None:
     import torch.distributed as dist
 
     from paper_1810_05291_b200 import binding as B
-    from paper_1810_05291_b200 import inputs
+    from paper_1810_05291_b200 import inputs, sharding
 
     world = int(os.environ.get("WORLD_SIZE", "1"))
     rank = int(os.environ.get("RANK", "0"))
@@ -313,10 +313,7 @@ def main() -> None:
         t1 = time.time()
     clocks = sampler.stop(t0, t1) if not args.profile else {"sm_mhz": None, "reasons": ["not sampled (--profile)"]}
 
-    if world > 1:
-        t = torch.tensor([ms_total], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_total = float(t.item())
+    ms_total = sharding.max_over_ranks(ms_total, dev)
     ms_step = ms_total / args.steps
     value = world * case.d / (ms_step * 1e-3)
 
@@ -341,10 +338,7 @@ def main() -> None:
         h1.record(stream)
         barrier()
         ms_e2e = h0.elapsed_time(h1)
-        if world > 1:
-            t = torch.tensor([ms_e2e], device=dev, dtype=torch.float64)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            ms_e2e = float(t.item())
+        ms_e2e = sharding.max_over_ranks(ms_e2e, dev)
         e2e = {"value": world * case.d / (ms_e2e / n_e2e * 1e-3), "unit": UNIT,
                "h2d_bytes_per_step": sum(h.numel() * h.element_size() for h in host),
                "d2h_bytes_per_step": hv.numel() * 4, "steps": n_e2e,
