@@ -142,6 +142,42 @@ int ss_fused_step_host(const void* const* host_grads, ss_dtype dt, void* const* 
                        uint32_t* host_vote_out, void* cuda_stream);
 
 /*
+ * ss_fused_step_host without any device memory from the caller or from an allocator.
+ * (The paper has no counterpart to this entry point; it exists for deployment.)
+ *
+ * Who needs it: a host program that cannot call cudaMalloc at the point where it wants a step.
+ * Typical cases are a process that has handed the whole device to a framework's caching
+ * allocator, so that a raw allocation fails or eats into that pool; a plug-in or a control loop
+ * whose rules forbid allocating after start-up, because cudaMalloc takes a device-wide lock and
+ * can stall every stream; and a sandboxed component that is given streams and buffers but not
+ * the right to create allocations. Such a caller cannot provide ss_fused_step_host's `staging`
+ * buffers, so here the staging area is a fixed array of SS_STATIC_STAGING_BYTES that is part of
+ * the library's device image: every GPU on which the library's CUDA module is loaded holds that
+ * much memory until the process exits.
+ *
+ *   host_grads      in      HOST array of M HOST pointers (pinned memory recommended), d elements each
+ *   momenta, param, vote_words_dev: caller-owned DEVICE memory as in ss_fused_step_host
+ *   host_vote_out   out     ceil(d/32) words of HOST memory, or NULL
+ *
+ * Limit: M * round_up(d * element size, 256) <= SS_STATIC_STAGING_BYTES. A larger request returns
+ * SS_ERR_UNSUPPORTED and enqueues nothing; split the coordinates into ranges and call once per range.
+ * The call itself performs no cudaMalloc, cudaFree or other allocating call.
+ * First call on a device: it looks up the device address of the staging array (once per device,
+ * with that device current) and keeps it. Make that first call during start-up, outside any
+ * stream capture.
+ * Sharing: all calls on a device use the same staging array, and it keeps whatever the last call
+ * left there. Every byte a call reads is first overwritten by that call's own copies, so nothing
+ * needs clearing; but two calls whose work overlaps on the GPU (different streams, no dependency)
+ * race on the array. Issue them on one stream or order them with events.
+ * Results are identical to ss_fused_step_host. Errors as for ss_fused_step_host.
+ */
+#define SS_STATIC_STAGING_BYTES (64u << 20)
+int ss_fused_step_host_static(const void* const* host_grads, ss_dtype dt, float* const* momenta,
+                              int M, int64_t d, float beta, uint64_t flip_mask, float* param,
+                              float lr, float weight_decay, uint32_t* vote_words_dev,
+                              uint32_t* host_vote_out, void* cuda_stream);
+
+/*
  * Launch-shape override for benchmarking sweeps (process-wide; not part of the method).
  *   key: "threads" (block size, multiple of 32 in [64, 1024], 0 = default) or
  *        "blocks_per_sm" (0 = one block per tile, the default; n > 0 = a persistent grid of

@@ -24,6 +24,7 @@ LIB_PATH = os.path.join(_HERE, "libsignsgd.so")
 SS_F32 = 0
 SS_BF16 = 1
 SS_MAX_WORKERS = 64
+SS_STATIC_STAGING_BYTES = 64 << 20
 
 SS_OK = 0
 SS_ERR_INVALID_ARG = -1
@@ -33,7 +34,7 @@ SS_ERR_CUDA = -4
 
 EXPORTS = ("ss_packed_words", "ss_status_string", "ss_last_cuda_error", "ss_sign_pack",
            "ss_majority_vote", "ss_signum_update", "ss_apply_vote", "ss_fused_step",
-           "ss_fused_step_host", "ss_set_launch_option")
+           "ss_fused_step_host", "ss_fused_step_host_static", "ss_set_launch_option")
 
 _lib = None
 
@@ -71,9 +72,11 @@ def lib() -> ctypes.CDLL:
     L.ss_apply_vote.argtypes = [vp, vp, i64, f32, f32, vp]
     L.ss_fused_step.argtypes = [vp, i32, vp, i32, i64, f32, u64, vp, f32, f32, vp, vp]
     L.ss_fused_step_host.argtypes = [vp, i32, vp, vp, i32, i64, f32, u64, vp, f32, f32, vp, vp, vp]
+    L.ss_fused_step_host_static.argtypes = [vp, i32, vp, i32, i64, f32, u64, vp, f32, f32, vp, vp, vp]
     L.ss_set_launch_option.argtypes = [ctypes.c_char_p, i32]
     for name in ("ss_sign_pack", "ss_majority_vote", "ss_signum_update", "ss_apply_vote",
-                 "ss_fused_step", "ss_fused_step_host", "ss_set_launch_option"):
+                 "ss_fused_step", "ss_fused_step_host", "ss_fused_step_host_static",
+                 "ss_set_launch_option"):
         getattr(L, name).restype = i32
     _lib = L
     return L
@@ -219,3 +222,40 @@ def ss_fused_step_host(host_grads: Sequence[torch.Tensor], staging: Sequence[tor
                                     float(lr), float(weight_decay),
                                     _words(vote_words_dev, d, "vote_words_dev"), hv, _stream(stream)),
            "ss_fused_step_host")
+
+
+def ss_fused_step_host_static(host_grads: Sequence[torch.Tensor],
+                              momenta: Optional[Sequence[torch.Tensor]], param: torch.Tensor,
+                              beta: float, lr: float, weight_decay: float, flip_mask: int,
+                              vote_words_dev: torch.Tensor, host_vote_out: Optional[torch.Tensor],
+                              stream=None) -> None:
+    """ss_fused_step_host for callers that may not allocate device memory: the gradients are
+    staged in a fixed array inside the library (at most SS_STATIC_STAGING_BYTES for all M workers
+    together), so no staging tensors are passed. The first call on a device looks up that array's
+    address; make it during start-up. Calls that overlap on the GPU race on the array."""
+    M = len(host_grads)
+    d = param.numel()
+    codes = {_dtype_code(g) for g in host_grads}
+    if len(codes) != 1:
+        raise TypeError("all gradients must share one dtype")
+    h_ptrs = []
+    for m, g in enumerate(host_grads):
+        if g.is_cuda or g.dim() != 1 or not g.is_contiguous() or g.numel() != d:
+            raise ValueError("host_grads[%d] must be a contiguous 1-D host tensor of d elements" % m)
+        h_ptrs.append(g.data_ptr())
+    v_arr = None
+    if momenta is not None:
+        if len(momenta) != M:
+            raise ValueError("need one momentum buffer per worker")
+        v_arr = _ptr_array([_dev(v, torch.float32, "momenta[%d]" % m, d) for m, v in enumerate(momenta)])
+    hv = None
+    if host_vote_out is not None:
+        if (host_vote_out.is_cuda or host_vote_out.dtype != torch.int32
+                or host_vote_out.numel() != ss_packed_words(d) or not host_vote_out.is_contiguous()):
+            raise ValueError("host_vote_out must be a contiguous host int32 tensor of ceil(d/32) words")
+        hv = host_vote_out.data_ptr()
+    _check(lib().ss_fused_step_host_static(_ptr_array(h_ptrs), codes.pop(), v_arr, M, d, float(beta),
+                                           int(flip_mask), _dev(param, torch.float32, "param"),
+                                           float(lr), float(weight_decay),
+                                           _words(vote_words_dev, d, "vote_words_dev"), hv,
+                                           _stream(stream)), "ss_fused_step_host_static")

@@ -49,6 +49,10 @@ inline bool overlap(const void* p, size_t n, const void* q, size_t m) {
 }
 
 }  // namespace
+
+// for the other translation units of the library
+int cuda_status_public(cudaError_t e) { return cuda_status(e); }
+
 }  // namespace ss
 
 using namespace ss;
