@@ -29,6 +29,14 @@ UNIT = "params/s"
 FALLBACK_HBM_GBS = 6650.0
 NOMINAL_HBM_GBS = 8000.0
 
+# DRAM bytes per coordinate (dram__bytes_read.sum + dram__bytes_write.sum) of the fused kernels,
+# from ncu captures at d = 8,388,608 (larger than L2; traffic is proportional to d because every
+# coordinate is touched exactly once). Keyed by (M, gradient bytes, momentum). An entry is
+# removed when its kernel changes until the counters are taken again.
+NCU_DRAM_BYTES_PER_COORD = {
+    (15, 4, True): (1.040216e9 + 487.84e6) / 8388608,
+}
+
 
 def make_case(name: str, d_override=None):
     from paper_1810_05291_b200 import inputs
@@ -61,6 +69,15 @@ def algorithmic_bytes(case) -> int:
     if case.beta is not None:
         per += case.M * 8
     return per * case.d
+
+
+def ncu_traffic(case):
+    """DRAM bytes of one launch of the fused kernel on this workload, scaled from the ncu capture
+    of a smaller case of the same kernel; None when no capture of that kernel is on record."""
+    import torch
+    key = (case.M, 4 if case.dtype == torch.float32 else 2, case.beta is not None)
+    per = NCU_DRAM_BYTES_PER_COORD.get(key)
+    return None if per is None else per * case.d
 
 
 def measured_peak():
@@ -218,6 +235,153 @@ def config_of(case, residency: str) -> dict:
             "entry_point": "ss_fused_step", "l2": residency}
 
 
+# ---- per-entry-point table: every kernel of the path on the named workloads ------------------
+
+def entry_bytes(case, entry: str) -> int:
+    """Algorithmic bytes of one call of an entry point (what the method must move): gradients
+    and fp32 state once each way they are needed, packed words at 4 bytes per 32 coordinates."""
+    import torch
+    gb = 4 if case.dtype == torch.float32 else 2
+    d, M = case.d, case.M
+    wb = ((d + 31) // 32) * 4
+    mom = case.beta is not None
+    if entry == "pack":
+        return gb * d + wb
+    if entry == "signum_update":
+        return (gb + 8) * d + wb
+    if entry == "vote":
+        return (M + 1) * wb
+    if entry == "apply":
+        return 8 * d + wb
+    if entry == "vote_apply":
+        return M * wb + 8 * d
+    if entry == "fused":
+        return algorithmic_bytes(case)
+    if entry == "chain":
+        per_worker = entry_bytes(case, "signum_update" if mom else "pack")
+        return M * per_worker + entry_bytes(case, "vote") + entry_bytes(case, "apply")
+    raise ValueError(entry)
+
+
+def time_launches(fn, n: int, warmup: int, stream, flush=None):
+    """Per-launch device times in ms: an event pair around every call of fn; when a flush buffer
+    (larger than L2) is given it is overwritten and then read back between calls, outside the
+    event pair, so that every call starts with an L2 that holds none of its data and no dirty
+    lines whose write-back would be charged to it."""
+    import torch
+
+    def cold():
+        flush.zero_()
+        flush.max()
+
+    for _ in range(warmup):
+        if flush is not None:
+            cold()
+        fn()
+    torch.cuda.synchronize()
+    pairs = []
+    for _ in range(n):
+        if flush is not None:
+            cold()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(stream)
+        fn()
+        b.record(stream)
+        pairs.append((a, b))
+    torch.cuda.synchronize()
+    return [a.elapsed_time(b) for a, b in pairs]
+
+
+def table_mode(args) -> None:
+    """--table: one JSON line per (workload, entry point) with median and best launch time,
+    achieved GB/s over the algorithmic bytes and the fraction of the measured copy bandwidth.
+    Every call starts from a cold L2 (a 512 MB buffer is overwritten and read between calls)."""
+    import torch
+
+    from paper_1810_05291_b200 import binding as B
+    from paper_1810_05291_b200 import inputs
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the library has no CPU path")
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(dev)
+    B.lib()
+    stream = torch.cuda.current_stream()
+    flush = torch.empty(512 << 20, dtype=torch.uint8, device=dev)
+    peak, peak_src = measured_peak()
+    if args.table == "named":
+        names = ["cfg1", "cfg2", "cfg3", "cfg4", "cfg4tie"]
+        entries = ["pack", "signum_update", "vote", "apply", "chain", "fused"]
+    elif args.table == "sweep":
+        names = ["sweep:%d:%d" % (d, M) for d in inputs.SWEEP_D for M in inputs.SWEEP_M]
+        entries = ["vote", "fused"]
+    else:
+        names = args.table.split(",")
+        entries = ["pack", "signum_update", "vote", "apply", "chain", "fused"]
+    rows = []
+    for name in names:
+        case = make_case(name, args.d)
+        mom = case.beta is not None
+        beta = case.beta if mom else 0.0
+        grads = inputs.gradients(case, dev, 0)
+        x = inputs.initial_params(case, dev)
+        moms = inputs.zero_momenta(case, dev)
+        W = B.ss_packed_words(case.d)
+        packed = [torch.zeros(W, dtype=torch.int32, device=dev) for _ in range(case.M)]
+        vote = torch.zeros(W, dtype=torch.int32, device=dev)
+        for m in range(case.M):
+            B.ss_sign_pack(grads[m], packed[m], stream)
+        turn = [0]
+
+        def call(entry):
+            m = turn[0] % case.M
+            turn[0] += 1
+            if entry == "pack":
+                B.ss_sign_pack(grads[m], packed[m], stream)
+            elif entry == "signum_update":
+                B.ss_signum_update(grads[m], moms[m], beta, packed[m], stream)
+            elif entry == "vote":
+                B.ss_majority_vote(packed, case.d, case.flip_mask, vote, stream)
+            elif entry == "apply":
+                B.ss_apply_vote(x, vote, case.lr, case.weight_decay, stream)
+            elif entry == "fused":
+                B.ss_fused_step(grads, moms, x, beta, case.lr, case.weight_decay, case.flip_mask,
+                                vote, stream)
+            elif entry == "chain":
+                for k in range(case.M):
+                    if mom:
+                        B.ss_signum_update(grads[k], moms[k], beta, packed[k], stream)
+                    else:
+                        B.ss_sign_pack(grads[k], packed[k], stream)
+                B.ss_majority_vote(packed, case.d, case.flip_mask, vote, stream)
+                B.ss_apply_vote(x, vote, case.lr, case.weight_decay, stream)
+
+        for entry in entries:
+            if entry == "signum_update" and not mom:
+                continue
+            ms = time_launches(lambda: call(entry), args.steps, max(3, args.warmup), stream, flush)
+            nbytes = entry_bytes(case, entry)
+            med, best = statistics.median(ms), min(ms)
+            row = {"table": args.table, "workload": case.name, "M": case.M, "d": case.d,
+                   "dtype": dtype_name(case), "entry": entry, "launches": len(ms),
+                   "ms_median": med, "ms_min": best, "algorithmic_bytes": nbytes,
+                   "gbs_median": nbytes / (med * 1e-3) / 1e9, "gbs_best": nbytes / (best * 1e-3) / 1e9,
+                   "frac_of_measured_copy": nbytes / (med * 1e-3) / 1e9 / peak,
+                   "params_per_s": case.d / (med * 1e-3), "l2": "cold (512 MB written then read before every call)",
+                   "peak": peak, "peak_source": peak_src}
+            rows.append(row)
+            print(json.dumps(row), flush=True)
+        del grads, x, moms, packed, vote
+        torch.cuda.empty_cache()
+    print("| workload | entry | ms (median) | ms (min) | algorithmic MB | GB/s (median) | of measured copy |")
+    print("|---|---|---|---|---|---|---|")
+    for r in rows:
+        print("| M=%d d=%d %s | %s | %.4f | %.4f | %.1f | %.0f | %.3f |" % (
+            r["M"], r["d"], "bf16" if r["dtype"].startswith("bf16") else "f32", r["entry"],
+            r["ms_median"], r["ms_min"], r["algorithmic_bytes"] / 1e6, r["gbs_median"],
+            r["frac_of_measured_copy"]))
+
+
 def main() -> None:
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -230,6 +394,9 @@ def main() -> None:
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--profile", action="store_true",
                     help="for runs under a profiler: no clock sampling, no end-to-end and CPU legs")
+    ap.add_argument("--table", default=None,
+                    help="time every entry point: 'named' (cfg1-4), 'sweep' (the d x M sweep) or a "
+                         "comma-separated list of workloads; one JSON line per row, then a table")
     ap.add_argument("--threads", type=int, default=0, help="launch-shape override: block size")
     ap.add_argument("--blocks-per-sm", type=int, default=0, help="launch-shape override")
     args = ap.parse_args()
@@ -240,6 +407,9 @@ def main() -> None:
 
     if args.impl == "reference":
         reference_arm(args)
+        return
+    if args.table:
+        table_mode(args)
         return
 
     import torch
@@ -358,7 +528,7 @@ def main() -> None:
             "hbm_gbs": achieved, "pct_of_nominal_8tbs": 100.0 * achieved / NOMINAL_HBM_GBS,
             "gradient_elements_per_s": value * case.M,
             "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
-                         "frac": achieved / peak, "traffic": None, "peak_source": peak_src,
+                         "frac": achieved / peak, "traffic": ncu_traffic(case), "peak_source": peak_src,
                          "kernel": "step_vec_kernel<M=%d,%s,momentum=%s,apply>" % (
                              case.M, "f32" if case.dtype == torch.float32 else "bf16",
                              "yes" if case.beta is not None else "no"),
