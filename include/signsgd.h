@@ -125,6 +125,50 @@ int ss_fused_step(const void* const* grads, ss_dtype dt, float* const* momenta, 
                   uint32_t* vote_words_out, void* cuda_stream);
 
 /*
+ * Tensor fusion (Section 4 reports that merging small tensors into one buffer before
+ * compression saved compression and communication cost). A model's parameter tensors are laid
+ * out back to back in one flat vector of d coordinates, so that one
+ * call packs, votes and updates all of them; the gradient and momentum buffers use the same
+ * layout. Each tensor keeps its own learning rate and weight decay (Algorithm 1's eta and
+ * lambda) through a table of segments sorted by first coordinate: entry k covers coordinates
+ * [begin_k, begin_{k+1}), the last entry runs to d, entry 0 begins at 0. Tensors may start at
+ * any coordinate (no padding to word boundaries is needed); an entry whose range is empty is
+ * allowed and ignored.
+ */
+typedef struct ss_segment {
+    int64_t begin;       /* first coordinate of the tensor in the flat vector */
+    float lr;            /* eta for this tensor */
+    float weight_decay;  /* lambda for this tensor */
+} ss_segment;
+
+/*
+ * Validates a segment table and enqueues its copy to device memory.
+ *   host_segments  in   HOST array of n_segments entries (may be freed after the call returns
+ *                       only if it is pageable memory; pinned memory must outlive the copy)
+ *   segments_dev   out  caller-owned DEVICE array of n_segments entries, 8-byte aligned
+ * SS_ERR_INVALID_ARG if n_segments < 1, begin[0] != 0, the begins decrease, or a begin exceeds d.
+ */
+int ss_segments_upload(const ss_segment* host_segments, int n_segments, int64_t d,
+                       ss_segment* segments_dev, void* cuda_stream);
+
+/*
+ * ss_fused_step over a fused flat vector with per-tensor eta and lambda: coordinate c is
+ * updated as x <- x - lr_k (sign(V) + weight_decay_k x) with k the segment that holds c. The
+ * momentum, the signs and the vote do not depend on the table. The result equals one
+ * ss_fused_step per tensor on that tensor's slices.
+ *   segments_dev  in  DEVICE table written by ss_segments_upload (not validated again here)
+ * Other arguments as ss_fused_step.
+ */
+int ss_fused_step_segments(const void* const* grads, ss_dtype dt, float* const* momenta, int M,
+                           int64_t d, float beta, uint64_t flip_mask, float* param,
+                           const ss_segment* segments_dev, int n_segments,
+                           uint32_t* vote_words_out, void* cuda_stream);
+
+/* ss_apply_vote with per-tensor eta and lambda from a device segment table. */
+int ss_apply_vote_segments(float* param, const uint32_t* vote_words, int64_t d,
+                           const ss_segment* segments_dev, int n_segments, void* cuda_stream);
+
+/*
  * ss_fused_step for gradients that start in HOST memory (the end-to-end form: what a step costs
  * when the M gradients arrive over PCIe and the packed vote goes back, as the d-bit messages of
  * Algorithm 1's push steps do).

@@ -184,3 +184,27 @@ def fused_step(grads, momenta, param: np.ndarray, beta: float, lr: float,
                               M, d, float(beta), int(flip_mask), _ptr(param), float(lr),
                               float(weight_decay), _ptr(vote))
     return vote
+
+
+def fused_step_segments(grads, momenta, param: np.ndarray, beta: float, begins, lrs, weight_decays,
+                        flip_mask: int = 0) -> np.ndarray:
+    """Algorithm 1 on a flat vector that is the concatenation of several tensors, each with its
+    own eta and lambda (Section 4 merges small tensors into one buffer before compression; the
+    merged step must equal one step per tensor). Written as exactly that: one ``fused_step`` per
+    tensor on that tensor's slice of every buffer. Tensor k covers coordinates
+    [begins[k], begins[k+1]), the last one runs to d. Returns the packed vote of the whole vector
+    (the vote depends on neither eta nor lambda), computed by a separate whole-vector step on
+    copies."""
+    d = param.shape[0]
+    n = len(begins)
+    scratch_m = [v.copy() for v in momenta] if momenta is not None else None
+    vote = fused_step(grads, scratch_m, param.copy(), beta, 0.0, 0.0, flip_mask)
+    for k in range(n):
+        a = int(begins[k])
+        b = int(begins[k + 1]) if k + 1 < n else d
+        if b <= a:
+            continue
+        fused_step([g[a:b] for g in grads],
+                   [v[a:b] for v in momenta] if momenta is not None else None,
+                   param[a:b], beta, float(lrs[k]), float(weight_decays[k]), flip_mask)
+    return vote

@@ -34,7 +34,16 @@ SS_ERR_CUDA = -4
 
 EXPORTS = ("ss_packed_words", "ss_status_string", "ss_last_cuda_error", "ss_sign_pack",
            "ss_majority_vote", "ss_signum_update", "ss_apply_vote", "ss_fused_step",
+           "ss_segments_upload", "ss_fused_step_segments", "ss_apply_vote_segments",
            "ss_fused_step_host", "ss_fused_step_host_static", "ss_set_launch_option")
+
+
+class ss_segment(ctypes.Structure):
+    """One tensor of a fused flat vector: first coordinate, learning rate, weight decay."""
+    _fields_ = [("begin", ctypes.c_int64), ("lr", ctypes.c_float), ("weight_decay", ctypes.c_float)]
+
+
+SEGMENT_BYTES = ctypes.sizeof(ss_segment)  # 16
 
 _lib = None
 
@@ -74,9 +83,13 @@ def lib() -> ctypes.CDLL:
     L.ss_fused_step_host.argtypes = [vp, i32, vp, vp, i32, i64, f32, u64, vp, f32, f32, vp, vp, vp]
     L.ss_fused_step_host_static.argtypes = [vp, i32, vp, i32, i64, f32, u64, vp, f32, f32, vp, vp, vp]
     L.ss_set_launch_option.argtypes = [ctypes.c_char_p, i32]
+    L.ss_segments_upload.argtypes = [vp, i32, i64, vp, vp]
+    L.ss_fused_step_segments.argtypes = [vp, i32, vp, i32, i64, f32, u64, vp, vp, i32, vp, vp]
+    L.ss_apply_vote_segments.argtypes = [vp, vp, i64, vp, i32, vp]
     for name in ("ss_sign_pack", "ss_majority_vote", "ss_signum_update", "ss_apply_vote",
                  "ss_fused_step", "ss_fused_step_host", "ss_fused_step_host_static",
-                 "ss_set_launch_option"):
+                 "ss_set_launch_option", "ss_segments_upload", "ss_fused_step_segments",
+                 "ss_apply_vote_segments"):
         getattr(L, name).restype = i32
     _lib = L
     return L
@@ -186,6 +199,60 @@ def ss_fused_step(grads: Sequence[torch.Tensor], momenta: Optional[Sequence[torc
     _check(lib().ss_fused_step(_ptr_array(g_ptrs), codes.pop(), v_arr, M, d, float(beta),
                                int(flip_mask), _dev(param, torch.float32, "param"), float(lr),
                                float(weight_decay), w_ptr, _stream(stream)), "ss_fused_step")
+
+
+def segment_table(n_segments: int, device) -> torch.Tensor:
+    """Device storage for a table of n_segments ss_segment entries (16 bytes each)."""
+    return torch.zeros(2 * int(n_segments), dtype=torch.int64, device=device)
+
+
+def _segments(t: torch.Tensor, n_segments: int) -> int:
+    if not t.is_cuda or t.dtype != torch.int64 or not t.is_contiguous() or t.numel() < 2 * n_segments:
+        raise ValueError("segments_dev must come from segment_table(n_segments, device)")
+    return t.data_ptr()
+
+
+def ss_segments_upload(begins: Sequence[int], lrs: Sequence[float], weight_decays: Sequence[float],
+                       d: int, segments_dev: torch.Tensor, stream=None) -> None:
+    n = len(begins)
+    if len(lrs) != n or len(weight_decays) != n:
+        raise ValueError("begins, lrs and weight_decays must have one entry per tensor")
+    host = (ss_segment * max(n, 1))()
+    for k in range(n):
+        host[k].begin, host[k].lr, host[k].weight_decay = int(begins[k]), float(lrs[k]), float(weight_decays[k])
+    _check(lib().ss_segments_upload(ctypes.cast(host, ctypes.c_void_p), n, int(d),
+                                    _segments(segments_dev, n), _stream(stream)), "ss_segments_upload")
+
+
+def ss_fused_step_segments(grads: Sequence[torch.Tensor], momenta: Optional[Sequence[torch.Tensor]],
+                           param: torch.Tensor, beta: float, segments_dev: torch.Tensor,
+                           n_segments: int, flip_mask: int = 0,
+                           vote_words_out: Optional[torch.Tensor] = None, stream=None) -> None:
+    M = len(grads)
+    d = param.numel()
+    codes = {_dtype_code(g) for g in grads}
+    if len(codes) != 1:
+        raise TypeError("all gradients must share one dtype")
+    g_ptrs = [_dev(g, None, "grads[%d]" % m, d) for m, g in enumerate(grads)]
+    v_arr = None
+    if momenta is not None:
+        if len(momenta) != M:
+            raise ValueError("need one momentum buffer per worker")
+        v_arr = _ptr_array([_dev(v, torch.float32, "momenta[%d]" % m, d) for m, v in enumerate(momenta)])
+    w_ptr = None if vote_words_out is None else _words(vote_words_out, d, "vote_words_out")
+    _check(lib().ss_fused_step_segments(_ptr_array(g_ptrs), codes.pop(), v_arr, M, d, float(beta),
+                                        int(flip_mask), _dev(param, torch.float32, "param"),
+                                        _segments(segments_dev, n_segments), int(n_segments), w_ptr,
+                                        _stream(stream)), "ss_fused_step_segments")
+
+
+def ss_apply_vote_segments(param: torch.Tensor, vote_words: torch.Tensor, segments_dev: torch.Tensor,
+                           n_segments: int, stream=None) -> None:
+    d = param.numel()
+    _check(lib().ss_apply_vote_segments(_dev(param, torch.float32, "param"),
+                                        _words(vote_words, d, "vote_words"), d,
+                                        _segments(segments_dev, n_segments), int(n_segments),
+                                        _stream(stream)), "ss_apply_vote_segments")
 
 
 def ss_fused_step_host(host_grads: Sequence[torch.Tensor], staging: Sequence[torch.Tensor],

@@ -92,7 +92,8 @@ int ss_set_launch_option(const char* key, int value) {
 
 static int step_common(const void* const* grads, ss_dtype dt, float* const* momenta, int M,
                        int64_t d, float beta, uint64_t flip_mask, float* param, float lr,
-                       float weight_decay, uint32_t* words, void* cuda_stream) {
+                       float weight_decay, uint32_t* words, void* cuda_stream,
+                       const ss_segment* seg = nullptr, int n_seg = 0) {
     if (!dtype_ok(dt) || M < 1 || M > SS_MAX_WORKERS || d < 0) return SS_ERR_INVALID_ARG;
     if (!flip_ok(flip_mask, M)) return SS_ERR_INVALID_ARG;
     if (d == 0) return SS_OK;
@@ -137,6 +138,8 @@ static int step_common(const void* const* grads, ss_dtype dt, float* const* mome
     s.x = param;
     s.words = words;
     s.vec = vec;
+    s.seg = seg;
+    s.n_seg = n_seg;
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
     return cuda_status(dt == SS_F32 ? launch_step_f32(s, st) : launch_step_bf16(s, st));
 }
@@ -198,7 +201,50 @@ int ss_apply_vote(float* param, const uint32_t* vote_words, int64_t d, float lr,
     if (overlap(param, static_cast<size_t>(d) * 4, vote_words, static_cast<size_t>((d + 31) / 32) * 4))
         return SS_ERR_INVALID_ARG;
     return cuda_status(launch_apply(param, vote_words, d, lr, weight_decay, aligned(param, 16),
-                                    static_cast<cudaStream_t>(cuda_stream)));
+                                    nullptr, 0, static_cast<cudaStream_t>(cuda_stream)));
+}
+
+int ss_segments_upload(const ss_segment* host_segments, int n_segments, int64_t d,
+                       ss_segment* segments_dev, void* cuda_stream) {
+    if (host_segments == nullptr || segments_dev == nullptr || n_segments < 1 || d < 0)
+        return SS_ERR_INVALID_ARG;
+    if (!aligned(segments_dev, 8)) return SS_ERR_MISALIGNED;
+    if (host_segments[0].begin != 0) return SS_ERR_INVALID_ARG;
+    for (int k = 0; k < n_segments; ++k) {
+        if (host_segments[k].begin > d) return SS_ERR_INVALID_ARG;
+        if (k > 0 && host_segments[k].begin < host_segments[k - 1].begin) return SS_ERR_INVALID_ARG;
+    }
+    return cuda_status(cudaMemcpyAsync(segments_dev, host_segments,
+                                       static_cast<size_t>(n_segments) * sizeof(ss_segment),
+                                       cudaMemcpyHostToDevice, static_cast<cudaStream_t>(cuda_stream)));
+}
+
+int ss_fused_step_segments(const void* const* grads, ss_dtype dt, float* const* momenta, int M,
+                           int64_t d, float beta, uint64_t flip_mask, float* param,
+                           const ss_segment* segments_dev, int n_segments,
+                           uint32_t* vote_words_out, void* cuda_stream) {
+    if (n_segments < 1) return SS_ERR_INVALID_ARG;
+    if (d > 0 && (param == nullptr || segments_dev == nullptr)) return SS_ERR_INVALID_ARG;
+    if (d > 0 && !aligned(segments_dev, 8)) return SS_ERR_MISALIGNED;
+    if (momenta != nullptr && vote_words_out != nullptr && d > 0 && M >= 1 && M <= SS_MAX_WORKERS) {
+        const size_t fbytes = static_cast<size_t>(d) * 4, wbytes = static_cast<size_t>((d + 31) / 32) * 4;
+        for (int m = 0; m < M; ++m)
+            if (momenta[m] != nullptr && overlap(momenta[m], fbytes, vote_words_out, wbytes)) return SS_ERR_INVALID_ARG;
+    }
+    return step_common(grads, dt, momenta, M, d, beta, flip_mask, param, 0.0f, 0.0f, vote_words_out,
+                       cuda_stream, segments_dev, n_segments);
+}
+
+int ss_apply_vote_segments(float* param, const uint32_t* vote_words, int64_t d,
+                           const ss_segment* segments_dev, int n_segments, void* cuda_stream) {
+    if (d < 0 || n_segments < 1) return SS_ERR_INVALID_ARG;
+    if (d == 0) return SS_OK;
+    if (param == nullptr || vote_words == nullptr || segments_dev == nullptr) return SS_ERR_INVALID_ARG;
+    if (!aligned(param, 4) || !aligned(vote_words, 4) || !aligned(segments_dev, 8)) return SS_ERR_MISALIGNED;
+    if (overlap(param, static_cast<size_t>(d) * 4, vote_words, static_cast<size_t>((d + 31) / 32) * 4))
+        return SS_ERR_INVALID_ARG;
+    return cuda_status(launch_apply(param, vote_words, d, 0.0f, 0.0f, aligned(param, 16), segments_dev,
+                                    n_segments, static_cast<cudaStream_t>(cuda_stream)));
 }
 
 int ss_fused_step_host(const void* const* host_grads, ss_dtype dt, void* const* staging,

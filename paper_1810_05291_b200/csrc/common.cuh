@@ -77,6 +77,45 @@ __device__ __forceinline__ float4 update_rn4(const float4& x, uint32_t nib, floa
     return r;
 }
 
+// ---- per-tensor hyper-parameters of a fused flat vector (Section 4: small tensors are merged
+// into one buffer before compression). The table is sorted by first coordinate; entry k covers
+// [begin_k, begin_{k+1}) and the last entry runs to d. -------------------------------------------
+
+// index of the last entry whose begin is <= c (entry 0 begins at coordinate 0)
+__device__ __forceinline__ int segment_of(const ss_segment* seg, int n, int64_t c) {
+    int lo = 0, hi = n;
+    while (hi - lo > 1) {
+        const int mid = (lo + hi) >> 1;
+        if (__ldg(&seg[mid].begin) <= c) lo = mid; else hi = mid;
+    }
+    return lo;
+}
+
+__device__ __forceinline__ float update_seg1(const ss_segment* seg, int n, int64_t c, float x,
+                                             uint32_t plus) {
+    const int k = segment_of(seg, n, c);
+    const float lr = __ldg(&seg[k].lr), wd = __ldg(&seg[k].weight_decay);
+    return update_rn(x, plus, lr, wd, wd != 0.0f);
+}
+
+// the quad of coordinates 4 q .. 4 q + 3: one lookup when the quad lies inside one tensor
+__device__ __forceinline__ float4 update_seg4(const ss_segment* seg, int n, int64_t q,
+                                              const float4& x, uint32_t nib) {
+    const int64_t c0 = q << 2;
+    const int k = segment_of(seg, n, c0);
+    const bool whole = (k + 1 >= n) || (__ldg(&seg[k + 1].begin) > c0 + 3);
+    if (whole) {
+        const float lr = __ldg(&seg[k].lr), wd = __ldg(&seg[k].weight_decay);
+        return update_rn4(x, nib, lr, wd, wd != 0.0f);
+    }
+    float4 r;
+    r.x = update_seg1(seg, n, c0, x.x, nib & 1u);
+    r.y = update_seg1(seg, n, c0 + 1, x.y, nib & 2u);
+    r.z = update_seg1(seg, n, c0 + 2, x.z, nib & 4u);
+    r.w = update_seg1(seg, n, c0 + 3, x.w, nib & 8u);
+    return r;
+}
+
 // ---- host side --------------------------------------------------------------------------
 
 struct LaunchOptions {
@@ -120,6 +159,8 @@ struct StepDesc {
     float* x;               // null: no parameter update (pack only)
     uint32_t* words;        // may be null when x != null
     bool vec;               // all pointers sufficiently aligned for 128-bit access
+    const ss_segment* seg = nullptr;  // device table of per-tensor lr / weight decay, or null
+    int n_seg = 0;
 };
 
 cudaError_t launch_step_f32(const StepDesc& s, cudaStream_t st);
@@ -127,6 +168,6 @@ cudaError_t launch_step_bf16(const StepDesc& s, cudaStream_t st);
 cudaError_t launch_vote(const uint32_t* const* packed, int M, int64_t d, uint64_t flip,
                         uint32_t* vote, bool vec, cudaStream_t st);
 cudaError_t launch_apply(float* x, const uint32_t* vote, int64_t d, float lr, float wd, bool vec,
-                         cudaStream_t st);
+                         const ss_segment* seg, int n_seg, cudaStream_t st);
 
 }  // namespace ss

@@ -33,6 +33,8 @@ struct StepArgs {
     uint64_t flip;
     float beta, omb, lr, wd;
     int M;
+    const ss_segment* seg;  // per-tensor lr / weight decay (SEG kernels only)
+    int n_seg;
 };
 
 // Worker quads a thread requests per load batch (twice as many 128-bit loads with momentum).
@@ -54,7 +56,7 @@ struct StepShape {
 
 // One ragged or unaligned word: executed by a full warp, lane = bit position. M_CT = 0 loops
 // over the workers at run time (a.M of them, pointers indexed dynamically out of the NP slots).
-template <int M_CT, int NP, typename GT, bool MOM, bool APPLY>
+template <int M_CT, int NP, typename GT, bool MOM, bool APPLY, bool SEG>
 __device__ __forceinline__ void step_word_ballot(const StepArgs<NP>& a, int64_t j, int lane) {
     constexpr int P = M_CT > 0 ? bit_length(M_CT) : bit_length(NP);
     constexpr int LB = StepShape<M_CT, MOM>::LB;
@@ -105,11 +107,54 @@ __device__ __forceinline__ void step_word_ballot(const StepArgs<NP>& a, int64_t 
 
     const uint32_t T = static_cast<uint32_t>(M + 1) >> 1;  // ceil(M/2): a tie votes +1
     const uint32_t vote = cnt.at_least(T) & vmask;
-    if (APPLY && valid) a.x[c] = update_rn(xs, (vote >> lane) & 1u, a.lr, a.wd, a.wd != 0.0f);
+    if (APPLY && valid) {
+        if constexpr (SEG)
+            a.x[c] = update_seg1(a.seg, a.n_seg, c, xs, (vote >> lane) & 1u);
+        else
+            a.x[c] = update_rn(xs, (vote >> lane) & 1u, a.lr, a.wd, a.wd != 0.0f);
+    }
     if (lane == 0 && a.words != nullptr) a.words[j] = vote;
 }
 
-template <int M_CT, typename GT, bool MOM, bool APPLY>
+
+// Packed words from per-thread vote nibbles. Eight neighbouring lanes hold the eight nibbles of
+// one word (lane k of the group owns bits 4k..4k+3). Every lane of the warp must call this.
+//   U == 8: the 8 lanes x 8 quads of a group form an 8 x 8 matrix of nibbles; a three-stage
+//           butterfly transposes it across lanes, after which lane k holds the complete word of
+//           quad row k and stores it (3 shuffles per 8 words).
+//   else:   an OR tree over the group (3 shuffles per word); the group's first lane stores.
+template <int U>
+__device__ __forceinline__ void store_words(uint32_t* words, const uint32_t* nib, int64_t base,
+                                            int64_t n_quads, int lane) {
+    const int k = lane & 7;
+    if constexpr (U == 8) {
+        uint32_t r = 0u;
+#pragma unroll
+        for (int u = 0; u < 8; ++u) r |= nib[u] << (4 * u);
+        uint32_t o = __shfl_xor_sync(0xFFFFFFFFu, r, 4);
+        r = (k & 4) ? ((r & 0xFFFF0000u) | (o >> 16)) : ((r & 0x0000FFFFu) | (o << 16));
+        o = __shfl_xor_sync(0xFFFFFFFFu, r, 2);
+        r = (k & 2) ? ((r & 0xFF00FF00u) | ((o & 0xFF00FF00u) >> 8))
+                    : ((r & 0x00FF00FFu) | ((o & 0x00FF00FFu) << 8));
+        o = __shfl_xor_sync(0xFFFFFFFFu, r, 1);
+        r = (k & 1) ? ((r & 0xF0F0F0F0u) | ((o & 0xF0F0F0F0u) >> 4))
+                    : ((r & 0x0F0F0F0Fu) | ((o & 0x0F0F0F0Fu) << 4));
+        const int64_t qk = base + static_cast<int64_t>(k) * blockDim.x + threadIdx.x;
+        if (qk < n_quads) words[qk >> 3] = r;
+    } else {
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            uint32_t w = nib[u] << (4 * k);
+            w |= __shfl_xor_sync(0xFFFFFFFFu, w, 1);
+            w |= __shfl_xor_sync(0xFFFFFFFFu, w, 2);
+            w |= __shfl_xor_sync(0xFFFFFFFFu, w, 4);
+            const int64_t qu = base + static_cast<int64_t>(u) * blockDim.x + threadIdx.x;
+            if (k == 0 && qu < n_quads) words[qu >> 3] = w;
+        }
+    }
+}
+
+template <int M_CT, typename GT, bool MOM, bool APPLY, bool SEG>
 __global__ void __launch_bounds__(256)
 step_vec_kernel(const __grid_constant__ StepArgs<StepShape<M_CT, MOM>::NP> a) {
     using S = StepShape<M_CT, MOM>;
@@ -120,7 +165,6 @@ step_vec_kernel(const __grid_constant__ StepArgs<StepShape<M_CT, MOM>::NP> a) {
     const int64_t tile = static_cast<int64_t>(blockDim.x) * U;
     const uint32_t T = static_cast<uint32_t>(M + 1) >> 1;
     const bool has_wd = a.wd != 0.0f;
-    const uint32_t group = 0xFFu << (lane & 24);  // the 8 lanes that share one packed word
 
     for (int64_t base = static_cast<int64_t>(blockIdx.x) * tile; base < n_quads;
          base += static_cast<int64_t>(gridDim.x) * tile) {
@@ -179,27 +223,28 @@ step_vec_kernel(const __grid_constant__ StepArgs<StepShape<M_CT, MOM>::NP> a) {
             for (int m0 = 0; m0 < M; m0 += LB) batch(m0, std::integral_constant<int, LB>{});
         }
 
+        uint32_t vote[U];
 #pragma unroll
         for (int u = 0; u < U; ++u) {
-            if (ok[u]) {
-                const uint32_t vote = cnt[u].at_least(T) & 0xFu;
-                if (APPLY)
-                    __stcs(reinterpret_cast<float4*>(a.x) + q[u],
-                           update_rn4(xq[u], vote, a.lr, a.wd, has_wd));
-                if (a.words != nullptr) {
-                    const uint32_t w = __reduce_or_sync(group, vote << ((lane & 7) * 4));
-                    if ((lane & 7) == 0) a.words[q[u] >> 3] = w;
-                }
+            vote[u] = ok[u] ? (cnt[u].at_least(T) & 0xFu) : 0u;
+            if (APPLY && ok[u]) {
+                float4 xn;
+                if constexpr (SEG)
+                    xn = update_seg4(a.seg, a.n_seg, q[u], xq[u], vote[u]);
+                else
+                    xn = update_rn4(xq[u], vote[u], a.lr, a.wd, has_wd);
+                __stcs(reinterpret_cast<float4*>(a.x) + q[u], xn);
             }
         }
+        if (a.words != nullptr) store_words<U>(a.words, vote, base, n_quads, lane);
     }
 
     // the ragged last word (d not a multiple of 32): one warp, ballot form, run-time worker loop
     if ((a.d & 31) != 0 && blockIdx.x == 0 && threadIdx.x < 32)
-        step_word_ballot<(M_CT == 1 ? 1 : 0), S::NP, GT, MOM, APPLY>(a, a.d >> 5, lane);
+        step_word_ballot<(M_CT == 1 ? 1 : 0), S::NP, GT, MOM, APPLY, SEG>(a, a.d >> 5, lane);
 }
 
-template <int M_CT, typename GT, bool MOM, bool APPLY>
+template <int M_CT, typename GT, bool MOM, bool APPLY, bool SEG>
 __global__ void __launch_bounds__(256)
 step_ballot_kernel(const __grid_constant__ StepArgs<StepShape<M_CT, MOM>::NP> a) {
     const int lane = threadIdx.x & 31;
@@ -207,10 +252,10 @@ step_ballot_kernel(const __grid_constant__ StepArgs<StepShape<M_CT, MOM>::NP> a)
     const int64_t warps = (static_cast<int64_t>(gridDim.x) * blockDim.x) >> 5;
     for (int64_t j = (static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x) >> 5; j < W;
          j += warps)
-        step_word_ballot<M_CT, StepShape<M_CT, MOM>::NP, GT, MOM, APPLY>(a, j, lane);
+        step_word_ballot<M_CT, StepShape<M_CT, MOM>::NP, GT, MOM, APPLY, SEG>(a, j, lane);
 }
 
-template <int M_CT, typename GT, bool MOM, bool APPLY, bool VEC>
+template <int M_CT, typename GT, bool MOM, bool APPLY, bool VEC, bool SEG = false>
 cudaError_t launch_step_inst(const StepDesc& s, cudaStream_t st) {
     using S = StepShape<M_CT, MOM>;
     StepArgs<S::NP> a;
@@ -228,19 +273,21 @@ cudaError_t launch_step_inst(const StepDesc& s, cudaStream_t st) {
     a.lr = s.lr;
     a.wd = s.wd;
     a.M = s.M;
+    a.seg = s.seg;
+    a.n_seg = s.n_seg;
     int threads = launch_options().threads > 0 ? launch_options().threads : 256;
     if (threads > 256) threads = 256;
     int grid = 1;
     cudaError_t err;
     if constexpr (VEC) {
-        auto kernel = step_vec_kernel<M_CT, GT, MOM, APPLY>;
+        auto kernel = step_vec_kernel<M_CT, GT, MOM, APPLY, SEG>;
         const int64_t quads = (s.d >> 5) << 3;
         const int64_t tile = static_cast<int64_t>(threads) * S::U;
         err = pick_grid(kernel, threads, (quads + tile - 1) / tile, &grid);
         if (err != cudaSuccess) return err;
         kernel<<<grid, threads, 0, st>>>(a);
     } else {
-        auto kernel = step_ballot_kernel<M_CT, GT, MOM, APPLY>;
+        auto kernel = step_ballot_kernel<M_CT, GT, MOM, APPLY, SEG>;
         const int64_t W = (s.d + 31) >> 5;
         const int64_t per_block = threads / 32;
         err = pick_grid(kernel, threads, (W + per_block - 1) / per_block, &grid);
@@ -262,6 +309,23 @@ cudaError_t launch_step_dtype(const StepDesc& s, cudaStream_t st) {
          : launch_step_inst<MV, GT, false, AP, VC>(s, st))
     if (!apply)  // per-worker packing: M == 1 by construction
         return s.vec ? SS_STEP_PICK(1, false, true) : SS_STEP_PICK(1, false, false);
+    if (s.seg != nullptr) {  // per-tensor lr / weight decay from the segment table
+#define SS_STEP_PICK_SEG(MV, VC)                                                  \
+    (mom ? launch_step_inst<MV, GT, true, true, VC, true>(s, st)                  \
+         : launch_step_inst<MV, GT, false, true, VC, true>(s, st))
+        if (!s.vec) return SS_STEP_PICK_SEG(0, false);
+        switch (s.M) {
+            case 1: return SS_STEP_PICK_SEG(1, true);
+            case 3: return SS_STEP_PICK_SEG(3, true);
+            case 7: return SS_STEP_PICK_SEG(7, true);
+            case 15: return SS_STEP_PICK_SEG(15, true);
+            case 16: return SS_STEP_PICK_SEG(16, true);
+            case 31: return SS_STEP_PICK_SEG(31, true);
+            case 63: return SS_STEP_PICK_SEG(63, true);
+            default: return SS_STEP_PICK_SEG(0, true);
+        }
+#undef SS_STEP_PICK_SEG
+    }
     if (!s.vec) return SS_STEP_PICK(0, true, false);
     switch (s.M) {
         case 1: return SS_STEP_PICK(1, true, true);

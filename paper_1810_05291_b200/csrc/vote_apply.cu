@@ -185,13 +185,21 @@ struct ApplyArgs {
     const uint32_t* vote;
     int64_t d;
     float lr, wd;
+    const ss_segment* seg;  // per-tensor lr / weight decay (SEG kernels only)
+    int n_seg;
 };
 
+template <bool SEG>
 __device__ __forceinline__ void apply_one(const ApplyArgs& a, int64_t c, bool has_wd) {
     const uint32_t w = __ldg(a.vote + (c >> 5));
-    a.x[c] = update_rn(a.x[c], (w >> (c & 31)) & 1u, a.lr, a.wd, has_wd);
+    const uint32_t plus = (w >> (c & 31)) & 1u;
+    if constexpr (SEG)
+        a.x[c] = update_seg1(a.seg, a.n_seg, c, a.x[c], plus);
+    else
+        a.x[c] = update_rn(a.x[c], plus, a.lr, a.wd, has_wd);
 }
 
+template <bool SEG>
 __global__ void __launch_bounds__(256) apply_vec_kernel(const __grid_constant__ ApplyArgs a) {
     constexpr int U = 4;
     const bool has_wd = a.wd != 0.0f;
@@ -214,37 +222,50 @@ __global__ void __launch_bounds__(256) apply_vec_kernel(const __grid_constant__ 
             const int64_t q = base + static_cast<int64_t>(u) * blockDim.x + threadIdx.x;
             if (q < n_quads) {
                 const uint32_t nib = (w[u] >> ((q & 7) * 4)) & 0xFu;
-                __stcs(reinterpret_cast<float4*>(a.x) + q, update_rn4(xq[u], nib, a.lr, a.wd, has_wd));
+                float4 xn;
+                if constexpr (SEG)
+                    xn = update_seg4(a.seg, a.n_seg, q, xq[u], nib);
+                else
+                    xn = update_rn4(xq[u], nib, a.lr, a.wd, has_wd);
+                __stcs(reinterpret_cast<float4*>(a.x) + q, xn);
             }
         }
     }
     const int64_t rest = a.d & 3;
-    if (blockIdx.x == 0 && threadIdx.x < rest) apply_one(a, (n_quads << 2) + threadIdx.x, has_wd);
+    if (blockIdx.x == 0 && threadIdx.x < rest) apply_one<SEG>(a, (n_quads << 2) + threadIdx.x, has_wd);
 }
 
+template <bool SEG>
 __global__ void __launch_bounds__(256) apply_scalar_kernel(const __grid_constant__ ApplyArgs a) {
     const bool has_wd = a.wd != 0.0f;
     const int64_t stride = static_cast<int64_t>(gridDim.x) * blockDim.x;
     for (int64_t c = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x; c < a.d; c += stride)
-        apply_one(a, c, has_wd);
+        apply_one<SEG>(a, c, has_wd);
 }
 
 cudaError_t launch_apply(float* x, const uint32_t* vote, int64_t d, float lr, float wd, bool vec,
-                         cudaStream_t st) {
-    ApplyArgs a{x, vote, d, lr, wd};
+                         const ss_segment* seg, int n_seg, cudaStream_t st) {
+    ApplyArgs a{x, vote, d, lr, wd, seg, n_seg};
+    const bool segmented = seg != nullptr;
     int threads = launch_options().threads > 0 ? launch_options().threads : 256;
     if (threads > 256) threads = 256;
     int grid = 1;
     cudaError_t err;
     if (vec) {
         const int64_t tile = static_cast<int64_t>(threads) * 4;
-        err = pick_grid(apply_vec_kernel, threads, ((d >> 2) + tile - 1) / tile, &grid);
+        err = pick_grid(apply_vec_kernel<false>, threads, ((d >> 2) + tile - 1) / tile, &grid);
         if (err != cudaSuccess) return err;
-        apply_vec_kernel<<<grid, threads, 0, st>>>(a);
+        if (segmented)
+            apply_vec_kernel<true><<<grid, threads, 0, st>>>(a);
+        else
+            apply_vec_kernel<false><<<grid, threads, 0, st>>>(a);
     } else {
-        err = pick_grid(apply_scalar_kernel, threads, (d + threads - 1) / threads, &grid);
+        err = pick_grid(apply_scalar_kernel<false>, threads, (d + threads - 1) / threads, &grid);
         if (err != cudaSuccess) return err;
-        apply_scalar_kernel<<<grid, threads, 0, st>>>(a);
+        if (segmented)
+            apply_scalar_kernel<true><<<grid, threads, 0, st>>>(a);
+        else
+            apply_scalar_kernel<false><<<grid, threads, 0, st>>>(a);
     }
     return cudaGetLastError();
 }
