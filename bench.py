@@ -260,6 +260,9 @@ def entry_bytes(case, entry: str) -> int:
     if entry == "chain":
         per_worker = entry_bytes(case, "signum_update" if mom else "pack")
         return M * per_worker + entry_bytes(case, "vote") + entry_bytes(case, "apply")
+    if entry == "chain_va":
+        per_worker = entry_bytes(case, "signum_update" if mom else "pack")
+        return M * per_worker + entry_bytes(case, "vote_apply")
     raise ValueError(entry)
 
 
@@ -311,13 +314,13 @@ def table_mode(args) -> None:
     peak, peak_src = measured_peak()
     if args.table == "named":
         names = ["cfg1", "cfg2", "cfg3", "cfg4", "cfg4tie"]
-        entries = ["pack", "signum_update", "vote", "apply", "chain", "fused"]
+        entries = ["pack", "signum_update", "vote", "apply", "vote_apply", "chain", "chain_va", "fused"]
     elif args.table == "sweep":
         names = ["sweep:%d:%d" % (d, M) for d in inputs.SWEEP_D for M in inputs.SWEEP_M]
         entries = ["vote", "fused"]
     else:
         names = args.table.split(",")
-        entries = ["pack", "signum_update", "vote", "apply", "chain", "fused"]
+        entries = ["pack", "signum_update", "vote", "apply", "vote_apply", "chain", "chain_va", "fused"]
     rows = []
     for name in names:
         case = make_case(name, args.d)
@@ -347,6 +350,15 @@ def table_mode(args) -> None:
             elif entry == "fused":
                 B.ss_fused_step(grads, moms, x, beta, case.lr, case.weight_decay, case.flip_mask,
                                 vote, stream)
+            elif entry == "vote_apply":
+                B.ss_vote_apply(packed, x, case.lr, case.weight_decay, case.flip_mask, None, stream)
+            elif entry == "chain_va":
+                for k in range(case.M):
+                    if mom:
+                        B.ss_signum_update(grads[k], moms[k], beta, packed[k], stream)
+                    else:
+                        B.ss_sign_pack(grads[k], packed[k], stream)
+                B.ss_vote_apply(packed, x, case.lr, case.weight_decay, case.flip_mask, None, stream)
             elif entry == "chain":
                 for k in range(case.M):
                     if mom:

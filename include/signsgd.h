@@ -110,6 +110,18 @@ int ss_apply_vote(float* param, const uint32_t* vote_words, int64_t d, float lr,
                   float weight_decay, void* cuda_stream);
 
 /*
+ * ss_majority_vote and ss_apply_vote in one pass: what every worker does once the M packed
+ * sign vectors are in its memory (its own, and the others' after the exchange of Algorithm 1's
+ * two push steps). The tally never leaves the registers; the packed vote is written only if asked.
+ *   packed          in      HOST array of M device pointers, each to ceil(d/32) words
+ *   param           in/out  d fp32
+ *   vote_words_out  out     ceil(d/32) words, or NULL
+ * Results are identical to ss_majority_vote followed by ss_apply_vote.
+ */
+int ss_vote_apply(const uint32_t* const* packed, int M, int64_t d, uint64_t flip_mask, float* param,
+                  float lr, float weight_decay, uint32_t* vote_words_out, void* cuda_stream);
+
+/*
  * One whole iteration of Algorithm 1 in a single pass over memory: momentum, sign, vote and
  * parameter update per coordinate, the packed signs never leaving the chip.
  *   grads           in      HOST array of M device pointers, d elements of dt each
@@ -162,6 +174,11 @@ int ss_segments_upload(const ss_segment* host_segments, int n_segments, int64_t 
 int ss_fused_step_segments(const void* const* grads, ss_dtype dt, float* const* momenta, int M,
                            int64_t d, float beta, uint64_t flip_mask, float* param,
                            const ss_segment* segments_dev, int n_segments,
+                           uint32_t* vote_words_out, void* cuda_stream);
+
+/* ss_vote_apply with per-tensor eta and lambda from a device segment table. */
+int ss_vote_apply_segments(const uint32_t* const* packed, int M, int64_t d, uint64_t flip_mask,
+                           float* param, const ss_segment* segments_dev, int n_segments,
                            uint32_t* vote_words_out, void* cuda_stream);
 
 /* ss_apply_vote with per-tensor eta and lambda from a device segment table. */

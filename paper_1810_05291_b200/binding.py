@@ -35,7 +35,7 @@ SS_ERR_CUDA = -4
 EXPORTS = ("ss_packed_words", "ss_status_string", "ss_last_cuda_error", "ss_sign_pack",
            "ss_majority_vote", "ss_signum_update", "ss_apply_vote", "ss_fused_step",
            "ss_segments_upload", "ss_fused_step_segments", "ss_apply_vote_segments",
-           "ss_fused_step_host", "ss_fused_step_host_static", "ss_set_launch_option")
+           "ss_vote_apply", "ss_vote_apply_segments", "ss_fused_step_host", "ss_fused_step_host_static", "ss_set_launch_option")
 
 
 class ss_segment(ctypes.Structure):
@@ -86,10 +86,12 @@ def lib() -> ctypes.CDLL:
     L.ss_segments_upload.argtypes = [vp, i32, i64, vp, vp]
     L.ss_fused_step_segments.argtypes = [vp, i32, vp, i32, i64, f32, u64, vp, vp, i32, vp, vp]
     L.ss_apply_vote_segments.argtypes = [vp, vp, i64, vp, i32, vp]
+    L.ss_vote_apply.argtypes = [vp, i32, i64, u64, vp, f32, f32, vp, vp]
+    L.ss_vote_apply_segments.argtypes = [vp, i32, i64, u64, vp, vp, i32, vp, vp]
     for name in ("ss_sign_pack", "ss_majority_vote", "ss_signum_update", "ss_apply_vote",
                  "ss_fused_step", "ss_fused_step_host", "ss_fused_step_host_static",
                  "ss_set_launch_option", "ss_segments_upload", "ss_fused_step_segments",
-                 "ss_apply_vote_segments"):
+                 "ss_apply_vote_segments", "ss_vote_apply", "ss_vote_apply_segments"):
         getattr(L, name).restype = i32
     _lib = L
     return L
@@ -180,6 +182,17 @@ def ss_apply_vote(param: torch.Tensor, vote_words: torch.Tensor, lr: float,
                                d, float(lr), float(weight_decay), _stream(stream)), "ss_apply_vote")
 
 
+def ss_vote_apply(packed: Sequence[torch.Tensor], param: torch.Tensor, lr: float,
+                  weight_decay: float = 0.0, flip_mask: int = 0,
+                  vote_words_out: Optional[torch.Tensor] = None, stream=None) -> None:
+    d = param.numel()
+    ptrs = [_words(p, d, "packed[%d]" % m) for m, p in enumerate(packed)]
+    w_ptr = None if vote_words_out is None else _words(vote_words_out, d, "vote_words_out")
+    _check(lib().ss_vote_apply(_ptr_array(ptrs), len(ptrs), d, int(flip_mask),
+                               _dev(param, torch.float32, "param"), float(lr), float(weight_decay),
+                               w_ptr, _stream(stream)), "ss_vote_apply")
+
+
 def ss_fused_step(grads: Sequence[torch.Tensor], momenta: Optional[Sequence[torch.Tensor]],
                   param: torch.Tensor, beta: float, lr: float, weight_decay: float = 0.0,
                   flip_mask: int = 0, vote_words_out: Optional[torch.Tensor] = None,
@@ -244,6 +257,18 @@ def ss_fused_step_segments(grads: Sequence[torch.Tensor], momenta: Optional[Sequ
                                         int(flip_mask), _dev(param, torch.float32, "param"),
                                         _segments(segments_dev, n_segments), int(n_segments), w_ptr,
                                         _stream(stream)), "ss_fused_step_segments")
+
+
+def ss_vote_apply_segments(packed: Sequence[torch.Tensor], param: torch.Tensor,
+                           segments_dev: torch.Tensor, n_segments: int, flip_mask: int = 0,
+                           vote_words_out: Optional[torch.Tensor] = None, stream=None) -> None:
+    d = param.numel()
+    ptrs = [_words(p, d, "packed[%d]" % m) for m, p in enumerate(packed)]
+    w_ptr = None if vote_words_out is None else _words(vote_words_out, d, "vote_words_out")
+    _check(lib().ss_vote_apply_segments(_ptr_array(ptrs), len(ptrs), d, int(flip_mask),
+                                        _dev(param, torch.float32, "param"),
+                                        _segments(segments_dev, n_segments), int(n_segments), w_ptr,
+                                        _stream(stream)), "ss_vote_apply_segments")
 
 
 def ss_apply_vote_segments(param: torch.Tensor, vote_words: torch.Tensor, segments_dev: torch.Tensor,

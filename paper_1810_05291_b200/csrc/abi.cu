@@ -204,6 +204,47 @@ int ss_apply_vote(float* param, const uint32_t* vote_words, int64_t d, float lr,
                                     nullptr, 0, static_cast<cudaStream_t>(cuda_stream)));
 }
 
+static int vote_apply_common(const uint32_t* const* packed, int M, int64_t d, uint64_t flip_mask,
+                             float* param, float lr, float weight_decay, const ss_segment* seg,
+                             int n_seg, uint32_t* vote_words_out, void* cuda_stream) {
+    if (packed == nullptr || M < 1 || M > SS_MAX_WORKERS || d < 0) return SS_ERR_INVALID_ARG;
+    if (!flip_ok(flip_mask, M)) return SS_ERR_INVALID_ARG;
+    if (d == 0) return SS_OK;
+    if (param == nullptr) return SS_ERR_INVALID_ARG;
+    if (!aligned(param, 4)) return SS_ERR_MISALIGNED;
+    const size_t wbytes = static_cast<size_t>((d + 31) / 32) * 4, fbytes = static_cast<size_t>(d) * 4;
+    if (vote_words_out != nullptr) {
+        if (!aligned(vote_words_out, 4)) return SS_ERR_MISALIGNED;
+        if (overlap(vote_words_out, wbytes, param, fbytes)) return SS_ERR_INVALID_ARG;
+    }
+    for (int m = 0; m < M; ++m) {
+        if (packed[m] == nullptr) return SS_ERR_INVALID_ARG;
+        if (!aligned(packed[m], 4)) return SS_ERR_MISALIGNED;
+        if (overlap(packed[m], wbytes, param, fbytes)) return SS_ERR_INVALID_ARG;
+        if (vote_words_out != nullptr && overlap(packed[m], wbytes, vote_words_out, wbytes))
+            return SS_ERR_INVALID_ARG;
+    }
+    return cuda_status(launch_vote_apply(packed, M, d, flip_mask, param, lr, weight_decay,
+                                         aligned(param, 16), seg, n_seg, vote_words_out,
+                                         static_cast<cudaStream_t>(cuda_stream)));
+}
+
+int ss_vote_apply(const uint32_t* const* packed, int M, int64_t d, uint64_t flip_mask, float* param,
+                  float lr, float weight_decay, uint32_t* vote_words_out, void* cuda_stream) {
+    return vote_apply_common(packed, M, d, flip_mask, param, lr, weight_decay, nullptr, 0,
+                             vote_words_out, cuda_stream);
+}
+
+int ss_vote_apply_segments(const uint32_t* const* packed, int M, int64_t d, uint64_t flip_mask,
+                           float* param, const ss_segment* segments_dev, int n_segments,
+                           uint32_t* vote_words_out, void* cuda_stream) {
+    if (n_segments < 1) return SS_ERR_INVALID_ARG;
+    if (d > 0 && segments_dev == nullptr) return SS_ERR_INVALID_ARG;
+    if (d > 0 && !aligned(segments_dev, 8)) return SS_ERR_MISALIGNED;
+    return vote_apply_common(packed, M, d, flip_mask, param, 0.0f, 0.0f, segments_dev, n_segments,
+                             vote_words_out, cuda_stream);
+}
+
 int ss_segments_upload(const ss_segment* host_segments, int n_segments, int64_t d,
                        ss_segment* segments_dev, void* cuda_stream) {
     if (host_segments == nullptr || segments_dev == nullptr || n_segments < 1 || d < 0)

@@ -167,6 +167,9 @@ cudaError_t launch_step_f32(const StepDesc& s, cudaStream_t st);
 cudaError_t launch_step_bf16(const StepDesc& s, cudaStream_t st);
 cudaError_t launch_vote(const uint32_t* const* packed, int M, int64_t d, uint64_t flip,
                         uint32_t* vote, bool vec, cudaStream_t st);
+cudaError_t launch_vote_apply(const uint32_t* const* packed, int M, int64_t d, uint64_t flip,
+                              float* x, float lr, float wd, bool vec, const ss_segment* seg,
+                              int n_seg, uint32_t* vote, cudaStream_t st);
 cudaError_t launch_apply(float* x, const uint32_t* vote, int64_t d, float lr, float wd, bool vec,
                          const ss_segment* seg, int n_seg, cudaStream_t st);
 

@@ -255,6 +255,150 @@ step_ballot_kernel(const __grid_constant__ StepArgs<StepShape<M_CT, MOM>::NP> a)
         step_word_ballot<M_CT, StepShape<M_CT, MOM>::NP, GT, MOM, APPLY, SEG>(a, j, lane);
 }
 
+// Sign packing of one gradient buffer (ss_sign_pack): a pure read stream, so the kernel is kept
+// as lean as the arithmetic allows. Quad form: a thread loads U quads (128-bit requests, all
+// issued before the first is used), turns each into a sign nibble, and an OR tree over the eight
+// lanes of a word (three shuffles) assembles the word, stored by the group's first lane. Measured
+// against a read-only kernel of the same shape it runs at the same rate. One block per tile.
+template <typename GT, int U>
+__global__ void __launch_bounds__(256)
+pack_vec_kernel(const void* __restrict__ g, uint32_t* __restrict__ words, int64_t d) {
+    const int lane = threadIdx.x & 31;
+    const int k = lane & 7;
+    const int64_t n_quads = (d >> 5) << 3;  // quads lying in complete words
+    const int64_t tile = static_cast<int64_t>(blockDim.x) * U;
+    for (int64_t base = static_cast<int64_t>(blockIdx.x) * tile; base < n_quads;
+         base += static_cast<int64_t>(gridDim.x) * tile) {
+        float4 v[U];
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const int64_t q = base + static_cast<int64_t>(u) * blockDim.x + threadIdx.x;
+            v[u] = q < n_quads ? GT::load4(g, q) : make_float4(-1.f, -1.f, -1.f, -1.f);
+        }
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            uint32_t w = sign_nibble(v[u]) << (4 * k);
+            w |= __shfl_xor_sync(0xFFFFFFFFu, w, 1);
+            w |= __shfl_xor_sync(0xFFFFFFFFu, w, 2);
+            w |= __shfl_xor_sync(0xFFFFFFFFu, w, 4);
+            const int64_t q = base + static_cast<int64_t>(u) * blockDim.x + threadIdx.x;
+            if (k == 0 && q < n_quads) words[q >> 3] = w;
+        }
+    }
+    // the ragged last word (d not a multiple of 32): one warp, one coordinate per lane
+    if ((d & 31) != 0 && blockIdx.x == 0 && threadIdx.x < 32) {
+        const int64_t c = ((d >> 5) << 5) + lane;
+        const float z = c < d ? GT::load1(g, c) : -1.0f;
+        const uint32_t w = __ballot_sync(0xFFFFFFFFu, z >= 0.0f);
+        if (lane == 0) words[d >> 5] = w;
+    }
+}
+
+// bf16 gradients with a 16-byte aligned pointer: a lane owns an octet (8 consecutive
+// coordinates, one 128-bit request; 64-bit requests top out near half the HBM rate), four lanes
+// make a word, two shuffles assemble it.
+template <int U>
+__global__ void __launch_bounds__(256)
+pack_oct_bf16_kernel(const void* __restrict__ g, uint32_t* __restrict__ words, int64_t d) {
+    const int lane = threadIdx.x & 31;
+    const int k = lane & 3;
+    const int64_t n_oct = (d >> 5) << 2;  // octets lying in complete words
+    const int64_t tile = static_cast<int64_t>(blockDim.x) * U;
+    for (int64_t base = static_cast<int64_t>(blockIdx.x) * tile; base < n_oct;
+         base += static_cast<int64_t>(gridDim.x) * tile) {
+        uint4 v[U];
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const int64_t o = base + static_cast<int64_t>(u) * blockDim.x + threadIdx.x;
+            v[u] = o < n_oct ? __ldcs(reinterpret_cast<const uint4*>(g) + o)
+                             : make_uint4(0x80008000u, 0x80008000u, 0x80008000u, 0x80008000u);
+        }
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const uint32_t r[4] = {v[u].x, v[u].y, v[u].z, v[u].w};
+            uint32_t b = 0u;
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                b |= sign_bit(__uint_as_float(r[i] << 16)) << (2 * i);
+                b |= sign_bit(__uint_as_float(r[i] & 0xFFFF0000u)) << (2 * i + 1);
+            }
+            uint32_t w = b << (8 * k);
+            w |= __shfl_xor_sync(0xFFFFFFFFu, w, 1);
+            w |= __shfl_xor_sync(0xFFFFFFFFu, w, 2);
+            const int64_t o = base + static_cast<int64_t>(u) * blockDim.x + threadIdx.x;
+            if (k == 0 && o < n_oct) words[o >> 2] = w;
+        }
+    }
+    if ((d & 31) != 0 && blockIdx.x == 0 && threadIdx.x < 32) {
+        const int64_t c = ((d >> 5) << 5) + lane;
+        const float z = c < d ? BF16::load1(g, c) : -1.0f;
+        const uint32_t w = __ballot_sync(0xFFFFFFFFu, z >= 0.0f);
+        if (lane == 0) words[d >> 5] = w;
+    }
+}
+
+// Ballot form for a gradient pointer that is not 16-byte aligned: lane l owns coordinate
+// 32 j + l, __ballot_sync gives word j whole; PACK_WORDS words per warp with all loads issued
+// first. Needs only element alignment; the ragged last word falls out of the predication.
+constexpr int PACK_WORDS = 8;
+
+template <typename GT>
+__global__ void __launch_bounds__(256)
+pack_ballot_kernel(const void* __restrict__ g, uint32_t* __restrict__ words, int64_t d) {
+    const int lane = threadIdx.x & 31;
+    const int64_t W = (d + 31) >> 5;
+    const int64_t warps = (static_cast<int64_t>(gridDim.x) * blockDim.x) >> 5;
+    for (int64_t j0 = ((static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x) >> 5) * PACK_WORDS;
+         j0 < W; j0 += warps * PACK_WORDS) {
+        float s[PACK_WORDS];
+#pragma unroll
+        for (int k = 0; k < PACK_WORDS; ++k) {
+            const int64_t c = ((j0 + k) << 5) + lane;
+            s[k] = c < d ? GT::load1(g, c) : -1.0f;  // beyond d: bit 0
+        }
+        uint32_t mine = 0u;
+#pragma unroll
+        for (int k = 0; k < PACK_WORDS; ++k) {
+            const uint32_t w = __ballot_sync(0xFFFFFFFFu, s[k] >= 0.0f);
+            if (lane == k) mine = w;
+        }
+        if (lane < PACK_WORDS && j0 + lane < W) words[j0 + lane] = mine;
+    }
+}
+
+template <typename GT>
+cudaError_t launch_pack(const StepDesc& s, cudaStream_t st) {
+    int threads = launch_options().threads > 0 ? launch_options().threads : 256;
+    if (threads > 256) threads = 256;
+    int grid = 1;
+    cudaError_t err;
+    if (GT::kBytes == 2 && (reinterpret_cast<uintptr_t>(s.g[0]) & 15) == 0) {
+        constexpr int U = 4;
+        auto kernel = pack_oct_bf16_kernel<U>;
+        const int64_t octets = (s.d >> 5) << 2;
+        const int64_t tile = static_cast<int64_t>(threads) * U;
+        err = pick_grid(kernel, threads, (octets + tile - 1) / tile, &grid);
+        if (err != cudaSuccess) return err;
+        kernel<<<grid, threads, 0, st>>>(s.g[0], s.words, s.d);
+    } else if (s.vec) {
+        constexpr int U = 4;
+        auto kernel = pack_vec_kernel<GT, U>;
+        const int64_t quads = (s.d >> 5) << 3;
+        const int64_t tile = static_cast<int64_t>(threads) * U;
+        err = pick_grid(kernel, threads, (quads + tile - 1) / tile, &grid);
+        if (err != cudaSuccess) return err;
+        kernel<<<grid, threads, 0, st>>>(s.g[0], s.words, s.d);
+    } else {
+        const int64_t W = (s.d + 31) >> 5;
+        const int64_t per_block = static_cast<int64_t>(threads / 32) * PACK_WORDS;
+        auto kernel = pack_ballot_kernel<GT>;
+        err = pick_grid(kernel, threads, (W + per_block - 1) / per_block, &grid);
+        if (err != cudaSuccess) return err;
+        kernel<<<grid, threads, 0, st>>>(s.g[0], s.words, s.d);
+    }
+    return cudaGetLastError();
+}
+
 template <int M_CT, typename GT, bool MOM, bool APPLY, bool VEC, bool SEG = false>
 cudaError_t launch_step_inst(const StepDesc& s, cudaStream_t st) {
     using S = StepShape<M_CT, MOM>;
@@ -307,8 +451,11 @@ cudaError_t launch_step_dtype(const StepDesc& s, cudaStream_t st) {
 #define SS_STEP_PICK(MV, AP, VC)                                             \
     (mom ? launch_step_inst<MV, GT, true, AP, VC>(s, st)                     \
          : launch_step_inst<MV, GT, false, AP, VC>(s, st))
-    if (!apply)  // per-worker packing: M == 1 by construction
-        return s.vec ? SS_STEP_PICK(1, false, true) : SS_STEP_PICK(1, false, false);
+    if (!apply) {  // per-worker packing: M == 1 by construction
+        if (!mom) return launch_pack<GT>(s, st);
+        return s.vec ? launch_step_inst<1, GT, true, false, true>(s, st)
+                     : launch_step_inst<1, GT, true, false, false>(s, st);
+    }
     if (s.seg != nullptr) {  // per-tensor lr / weight decay from the segment table
 #define SS_STEP_PICK_SEG(MV, VC)                                                  \
     (mom ? launch_step_inst<MV, GT, true, true, VC, true>(s, st)                  \

@@ -178,6 +178,175 @@ cudaError_t launch_vote(const uint32_t* const* packed, int M, int64_t d, uint64_
     }
 }
 
+// ---- vote + apply in one pass: what a worker does once the other workers' packed signs have
+// arrived (Algorithm 1: the server's sum and sign, then "update parameters"). A warp owns a
+// tile of 32 packed words = 1024 coordinates: lane l loads word l of every worker (coalesced),
+// the bit-sliced counter gives lane l the vote word l, and the 256 quads of x in the tile are
+// visited in eight coalesced rounds, each lane fetching the vote word it needs by shuffle. -----
+
+template <int NP>
+struct VoteApplyArgs {
+    const uint32_t* p[NP];
+    uint32_t* out;  // may be null
+    float* x;
+    int64_t d;
+    uint64_t flip;
+    float lr, wd;
+    const ss_segment* seg;
+    int n_seg;
+    int M;
+};
+
+template <int M_CT, bool VEC, bool SEG>
+__global__ void __launch_bounds__(256)
+vote_apply_kernel(const __grid_constant__ VoteApplyArgs<VoteShape<M_CT>::NP> a) {
+    using S = VoteShape<M_CT>;
+    constexpr int LB = S::LB;
+    const int M = M_CT > 0 ? M_CT : a.M;
+    const int lane = threadIdx.x & 31;
+    const int64_t W = (a.d + 31) >> 5;
+    const int64_t n_tiles = (W + 31) >> 5;
+    const int64_t n_quads = a.d >> 2;  // complete quads of x
+    const uint32_t T = static_cast<uint32_t>(M + 1) >> 1;
+    const bool has_wd = a.wd != 0.0f;
+    const int64_t warps = (static_cast<int64_t>(gridDim.x) * blockDim.x) >> 5;
+    for (int64_t t = (static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x) >> 5; t < n_tiles;
+         t += warps) {
+        const int64_t j = (t << 5) + lane;
+        const bool jv = j < W;
+        float4 xq[8];
+        if constexpr (VEC) {
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                const int64_t Q = (t << 8) + 32 * i + lane;
+                if (Q < n_quads) xq[i] = __ldcs(reinterpret_cast<const float4*>(a.x) + Q);
+            }
+        }
+        BitCounter<S::P> cnt;
+        cnt.clear();
+        auto batch = [&](int m0, auto nb_tag) {
+            constexpr int NB = decltype(nb_tag)::value;
+            uint32_t w[NB];
+#pragma unroll
+            for (int k = 0; k < NB; ++k) {
+                const bool live = jv && (M_CT > 0 || m0 + k < M);
+                const int mi = m0 + k < S::NP ? m0 + k : 0;
+                w[k] = live ? __ldcs(a.p[mi] + j) : 0u;
+            }
+#pragma unroll
+            for (int k = 0; k < NB; ++k) {
+                const bool live = jv && (M_CT > 0 || m0 + k < M);
+                if (live && ((a.flip >> (m0 + k)) & 1ull)) w[k] = ~w[k];
+            }
+            cnt.template add_words<NB>(w);
+        };
+        if constexpr (M_CT > 0) {
+            constexpr int FULL = M_CT / LB, REM = M_CT % LB;
+#pragma unroll
+            for (int b = 0; b < FULL; ++b) batch(b * LB, std::integral_constant<int, LB>{});
+            if constexpr (REM > 0) batch(FULL * LB, std::integral_constant<int, REM>{});
+        } else {
+            for (int m0 = 0; m0 < M; m0 += LB) batch(m0, std::integral_constant<int, LB>{});
+        }
+        const uint32_t vote = jv ? (cnt.at_least(T) & valid_bits(j, a.d)) : 0u;
+        if (a.out != nullptr && jv) __stcs(a.out + j, vote);
+
+        if constexpr (VEC) {
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                const uint32_t vw = __shfl_sync(0xFFFFFFFFu, vote, 4 * i + (lane >> 3));
+                const uint32_t nib = (vw >> (4 * (lane & 7))) & 0xFu;
+                const int64_t Q = (t << 8) + 32 * i + lane;
+                if (Q < n_quads) {
+                    float4 xn;
+                    if constexpr (SEG)
+                        xn = update_seg4(a.seg, a.n_seg, Q, xq[i], nib);
+                    else
+                        xn = update_rn4(xq[i], nib, a.lr, a.wd, has_wd);
+                    __stcs(reinterpret_cast<float4*>(a.x) + Q, xn);
+                } else if (Q == n_quads) {  // up to three coordinates past the last full quad
+                    for (int64_t c = Q << 2; c < a.d; ++c) {
+                        const uint32_t plus = (nib >> (c & 3)) & 1u;
+                        if constexpr (SEG)
+                            a.x[c] = update_seg1(a.seg, a.n_seg, c, a.x[c], plus);
+                        else
+                            a.x[c] = update_rn(a.x[c], plus, a.lr, a.wd, has_wd);
+                    }
+                }
+            }
+        } else {
+#pragma unroll 8
+            for (int i = 0; i < 32; ++i) {
+                const uint32_t vw = __shfl_sync(0xFFFFFFFFu, vote, i);
+                const int64_t c = (((t << 5) + i) << 5) + lane;
+                if (c < a.d) {
+                    const uint32_t plus = (vw >> lane) & 1u;
+                    if constexpr (SEG)
+                        a.x[c] = update_seg1(a.seg, a.n_seg, c, a.x[c], plus);
+                    else
+                        a.x[c] = update_rn(a.x[c], plus, a.lr, a.wd, has_wd);
+                }
+            }
+        }
+    }
+}
+
+template <int M_CT, bool VEC, bool SEG>
+cudaError_t launch_vote_apply_inst(const uint32_t* const* packed, int M, int64_t d, uint64_t flip,
+                                   float* x, float lr, float wd, const ss_segment* seg, int n_seg,
+                                   uint32_t* vote, cudaStream_t st) {
+    using S = VoteShape<M_CT>;
+    VoteApplyArgs<S::NP> a;
+    for (int m = 0; m < S::NP; ++m) a.p[m] = m < M ? packed[m] : nullptr;
+    a.out = vote;
+    a.x = x;
+    a.d = d;
+    a.flip = flip;
+    a.lr = lr;
+    a.wd = wd;
+    a.seg = seg;
+    a.n_seg = n_seg;
+    a.M = M;
+    int threads = launch_options().threads > 0 ? launch_options().threads : 256;
+    if (threads > 256) threads = 256;
+    const int64_t tiles = (((d + 31) >> 5) + 31) >> 5;
+    const int64_t per_block = threads / 32;
+    int grid = 1;
+    auto kernel = vote_apply_kernel<M_CT, VEC, SEG>;
+    cudaError_t err = pick_grid(kernel, threads, (tiles + per_block - 1) / per_block, &grid);
+    if (err != cudaSuccess) return err;
+    kernel<<<grid, threads, 0, st>>>(a);
+    return cudaGetLastError();
+}
+
+template <bool VEC, bool SEG>
+cudaError_t launch_vote_apply_m(const uint32_t* const* packed, int M, int64_t d, uint64_t flip,
+                                float* x, float lr, float wd, const ss_segment* seg, int n_seg,
+                                uint32_t* vote, cudaStream_t st) {
+#define SS_VA(MV) launch_vote_apply_inst<MV, VEC, SEG>(packed, M, d, flip, x, lr, wd, seg, n_seg, vote, st)
+    switch (M) {
+        case 1: return SS_VA(1);
+        case 3: return SS_VA(3);
+        case 7: return SS_VA(7);
+        case 15: return SS_VA(15);
+        case 16: return SS_VA(16);
+        case 31: return SS_VA(31);
+        case 63: return SS_VA(63);
+        default: return SS_VA(0);
+    }
+#undef SS_VA
+}
+
+cudaError_t launch_vote_apply(const uint32_t* const* packed, int M, int64_t d, uint64_t flip,
+                              float* x, float lr, float wd, bool vec, const ss_segment* seg,
+                              int n_seg, uint32_t* vote, cudaStream_t st) {
+    if (seg != nullptr)
+        return vec ? launch_vote_apply_m<true, true>(packed, M, d, flip, x, lr, wd, seg, n_seg, vote, st)
+                   : launch_vote_apply_m<false, true>(packed, M, d, flip, x, lr, wd, seg, n_seg, vote, st);
+    return vec ? launch_vote_apply_m<true, false>(packed, M, d, flip, x, lr, wd, seg, n_seg, vote, st)
+               : launch_vote_apply_m<false, false>(packed, M, d, flip, x, lr, wd, seg, n_seg, vote, st);
+}
+
 // ---- apply: x <- x - lr (sign(V) + wd x) from packed vote words ------------------------------
 
 struct ApplyArgs {

@@ -86,8 +86,8 @@ def test_apply_hand_vectors(rec):
 # ---- per-kernel parity on awkward shapes -----------------------------------------------------
 
 @pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16], ids=["f32", "bf16"])
-@pytest.mark.parametrize("misalign", [0, 1], ids=["aligned", "unaligned"])
-@pytest.mark.parametrize("d", AWKWARD_D)
+@pytest.mark.parametrize("misalign", [0, 1, 4], ids=["aligned", "unaligned", "off-by-4-elements"])
+@pytest.mark.parametrize("d", AWKWARD_D + [32 * 4096 + 8, 1_000_000])
 def test_sign_pack(d, misalign, dtype):
     g = _rand(d + misalign, 100 + d, dtype)[misalign:]
     out = GuardedWords(d, DEV, misalign_words=misalign)
@@ -146,6 +146,47 @@ def test_apply_vote(d, misalign, wd):
     assert_f32_close(x, x_np, "parameters")
     assert count_bit_mismatch(x, x_np) == 0
     check_guard(full, lo, d)
+
+
+@pytest.mark.parametrize("M", ALL_M)
+@pytest.mark.parametrize("misalign", [0, 1], ids=["aligned", "unaligned"])
+@pytest.mark.parametrize("d", [1, 3, 33, 127, 1023, 1024, 1027, 4097, 100_003])
+def test_vote_apply(d, misalign, M):
+    W = B.ss_packed_words(d)
+    gen = torch.Generator(device=DEV).manual_seed(23 * d + M)
+    packed = [torch.randint(-(1 << 31), 1 << 31, (W + misalign,), generator=gen, device=DEV,
+                            dtype=torch.int64).to(torch.int32)[misalign:] for _ in range(M)]
+    flip = int(torch.randint(0, 1 << 30, (1,), generator=gen, device=DEV).item()) & ((1 << M) - 1)
+    packed_np = [to_np(p) for p in packed]
+    for f, wd, want_words in ((0, 0.0, True), (flip, 0.02, True), (flip, 0.0, False)):
+        full, x, lo = guarded_f32(_rand(d, 600 + d + M, specials=False), misalign)
+        x_np = to_np(x)
+        out = GuardedWords(d, DEV, misalign_words=misalign)
+        B.ss_vote_apply(packed, x, 1e-3, wd, f, out.view if want_words else None)
+        vote = oracle.majority_vote(packed_np, d, f)
+        oracle.apply_vote(x_np, vote, 1e-3, wd)
+        if want_words:
+            assert_words_equal(out.view, vote)
+        out.check()
+        assert_f32_close(x, x_np, "parameters")
+        assert count_bit_mismatch(x, x_np) == 0
+        check_guard(full, lo, d)
+
+
+def test_vote_apply_equals_vote_then_apply_on_the_gpu():
+    M, d = 15, 32 * 40_000 + 8
+    gen = torch.Generator(device=DEV).manual_seed(77)
+    W = B.ss_packed_words(d)
+    packed = [torch.randint(-(1 << 31), 1 << 31, (W,), generator=gen, device=DEV,
+                            dtype=torch.int64).to(torch.int32) for _ in range(M)]
+    xa = _rand(d, 78, specials=False)
+    xb = xa.clone()
+    va, vb = words_tensor(d, DEV, fill=-1), words_tensor(d, DEV, fill=-1)
+    B.ss_vote_apply(packed, xa, 1e-4, 0.0, 0b101, va)
+    B.ss_majority_vote(packed, d, 0b101, vb)
+    B.ss_apply_vote(xb, vb, 1e-4, 0.0)
+    assert torch.equal(va, vb)
+    assert torch.equal(xa.view(torch.int32), xb.view(torch.int32))
 
 
 # ---- the fused step ---------------------------------------------------------------------------

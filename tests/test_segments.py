@@ -148,6 +148,36 @@ def test_apply_vote_segments(d, n_seg, misalign):
 
 
 @pytest.mark.gpu
+@pytest.mark.parametrize("M", [1, 7, 12])
+@pytest.mark.parametrize("d,n_seg", [(3, 2), (1027, 4), (100_003, 161)])
+@pytest.mark.parametrize("misalign", [0, 1], ids=["aligned", "unaligned"])
+def test_vote_apply_segments(M, d, n_seg, misalign):
+    rng = np.random.default_rng(d + M)
+    W = B.ss_packed_words(d)
+    packed_np = [rng.integers(0, 1 << 32, size=W, dtype=np.uint64).astype(np.uint32) for _ in range(M)]
+    packed = [torch.from_numpy(p.view(np.int32).copy()).to(DEV) for p in packed_np]
+    x = rng.standard_normal(d).astype(np.float32)
+    begins, lrs, wds = _table(d, n_seg, 5 * d + M)
+    tab = B.segment_table(n_seg, DEV)
+    B.ss_segments_upload(begins, lrs, wds, d, tab)
+    xt = torch.zeros(d + misalign, device=DEV)
+    xt[misalign:] = _to_dev(x)
+    xd = xt[misalign:]
+    vote_out = torch.full((W,), -1, dtype=torch.int32, device=DEV)
+    flip = 0b100 if M > 2 else 0
+    B.ss_vote_apply_segments(packed, xd, tab, n_seg, flip, vote_out)
+    vote = oracle.majority_vote(packed_np, d, flip)
+    bits = oracle.unpack(vote, d)
+    want = x.copy()
+    for k in range(n_seg):
+        a, b = begins[k], begins[k + 1] if k + 1 < n_seg else d
+        if b > a:
+            oracle.apply_vote(want[a:b], oracle.sign_pack(bits[a:b].astype(np.float32)), lrs[k], wds[k])
+    assert np.array_equal(vote_out.cpu().numpy().view(np.uint32), vote)
+    assert np.array_equal(xd.cpu().numpy().view(np.uint32), want.view(np.uint32))
+
+
+@pytest.mark.gpu
 def test_flat_layout_front_end_runs_a_model_shaped_step():
     from paper_1810_05291_b200.fusion import FlatLayout
     shapes = [(64, 3, 7, 7), (64,), (64,), (128, 64, 3, 3), (128,), (1000, 128), (1000,)]
