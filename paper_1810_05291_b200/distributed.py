@@ -1,0 +1,160 @@
+"""One worker of Algorithm 1 per GPU: the exchange of packed signs between the kernels.
+
+With the M workers on M GPUs, an iteration of Algorithm 1 has exactly one exchange step: every
+worker pushes the d sign bits of its momentum and receives the d bits of the vote (2 M d bits
+per iteration over the whole system, Appendix B). Two layouts of that exchange are provided,
+both carried by ``torch.distributed`` collectives (NCCL on GPUs); received words always land in
+this GPU's own memory before a kernel reads them.
+
+``allgather``  every worker receives all M packed vectors (d/8 bytes from each peer) and runs
+               ``ss_vote_apply`` locally: one collective, (M-1) d/8 bytes received per worker.
+``sharded``    the parameter server split across the workers (the future-work item of the
+               paper's discussion section): worker r is the server for the r-th slice of the
+               words. An all-to-all brings every worker's slice r to worker r, which votes on
+               it (``ss_majority_vote``); an all-gather returns the voted slices, and
+               ``ss_apply_vote`` updates the parameters: about 2 (M-1)/M d/8 bytes per worker.
+
+``PackedExchange`` holds the buffers and the slice arithmetic and works on any device (the
+multi-process CPU tests drive it over gloo); ``MajorityVoteWorker`` adds the kernels and needs
+CUDA tensors. There is no CPU path for the arithmetic.
+"""
+
+from __future__ import annotations
+
+from typing import List, Optional
+
+import torch
+import torch.distributed as dist
+
+
+def packed_words(d: int) -> int:
+    return (int(d) + 31) // 32
+
+
+class PackedExchange:
+    """Buffers and collectives for the packed sign words of one worker."""
+
+    def __init__(self, d: int, world: int, rank: int, device, mode: str = "allgather", group=None,
+                 collectives=None):
+        if mode not in ("allgather", "sharded"):
+            raise ValueError("mode must be 'allgather' or 'sharded'")
+        if world < 1 or not 0 <= rank < world or d < 0:
+            raise ValueError("bad world/rank/d")
+        self.d, self.world, self.rank, self.mode, self.group = int(d), world, rank, mode, group
+        self.coll = collectives if collectives is not None else dist
+        self.W = packed_words(d)
+        self.slice_words = -(-max(self.W, 1) // world)      # words per server slice
+        self.W_pad = self.slice_words * world               # local buffer, padded with zero words
+        kw = dict(dtype=torch.int32, device=device)
+        self.local = torch.zeros(self.W_pad, **kw)          # this worker's packed sign(v)
+        if mode == "allgather":
+            self.gathered = torch.zeros(world * self.W_pad, **kw)
+        else:
+            self.recv = torch.zeros(world * self.slice_words, **kw)
+            self.vote_slice = torch.zeros(self.slice_words, **kw)
+            self.vote_pad = torch.zeros(self.W_pad, **kw)
+
+    # ---- views ------------------------------------------------------------------------------
+    def local_words(self) -> torch.Tensor:
+        """Where the worker-side kernel writes this worker's ceil(d/32) words."""
+        return self.local[: self.W]
+
+    def worker_rows(self) -> List[torch.Tensor]:
+        """allgather mode, after gather(): worker m's packed vector, m = 0..M-1."""
+        return [self.gathered[m * self.W_pad: m * self.W_pad + self.W] for m in range(self.world)]
+
+    def slice_coordinates(self) -> int:
+        """sharded mode: how many of the d coordinates fall in this worker's server slice."""
+        first = 32 * self.rank * self.slice_words
+        return max(0, min(self.d - first, 32 * self.slice_words))
+
+    def slice_rows(self) -> List[torch.Tensor]:
+        """sharded mode, after scatter_slices(): worker m's words of this worker's slice."""
+        n = packed_words(self.slice_coordinates())
+        return [self.recv[m * self.slice_words: m * self.slice_words + n] for m in range(self.world)]
+
+    def slice_vote(self) -> torch.Tensor:
+        """sharded mode: where the server-side kernel writes this slice's vote words."""
+        return self.vote_slice[: packed_words(self.slice_coordinates())]
+
+    def vote_words(self) -> torch.Tensor:
+        """sharded mode, after gather_vote(): the packed vote of the whole vector."""
+        return self.vote_pad[: self.W]
+
+    # ---- collectives ------------------------------------------------------------------------
+    def gather(self) -> None:
+        self.coll.all_gather_into_tensor(self.gathered, self.local, group=self.group)
+
+    def scatter_slices(self) -> None:
+        self.coll.all_to_all_single(self.recv, self.local, group=self.group)
+
+    def gather_vote(self) -> None:
+        self.coll.all_gather_into_tensor(self.vote_pad, self.vote_slice, group=self.group)
+
+    def bytes_received_per_step(self) -> int:
+        """Bytes this worker receives from its peers per iteration (excludes its own share)."""
+        if self.mode == "allgather":
+            return (self.world - 1) * self.W_pad * 4
+        return 2 * (self.world - 1) * self.slice_words * 4
+
+
+class MajorityVoteWorker:
+    """Algorithm 1 as seen from one worker: momentum and sign packing of the local gradient,
+    the exchange, then vote and parameter update. State (x, v) lives on this worker's GPU."""
+
+    def __init__(self, param: torch.Tensor, beta: Optional[float], lr: float,
+                 weight_decay: float = 0.0, mode: str = "allgather", group=None, world=None,
+                 rank=None, collectives=None):
+        from . import binding as B
+        if not param.is_cuda:
+            raise ValueError("MajorityVoteWorker needs CUDA tensors: the arithmetic has no CPU path")
+        B.lib()
+        self.B = B
+        self.x = param
+        self.d = param.numel()
+        self.beta, self.lr, self.weight_decay = beta, float(lr), float(weight_decay)
+        if world is None:
+            world = dist.get_world_size(group)
+        if rank is None:
+            rank = dist.get_rank(group)
+        self.momentum = torch.zeros_like(param) if beta is not None else None
+        self.ex = PackedExchange(self.d, world, rank, param.device, mode, group, collectives)
+        self.vote = torch.zeros(self.ex.W, dtype=torch.int32, device=param.device)
+
+    def pack_local(self, grad: torch.Tensor, stream=None) -> None:
+        """Worker side: v <- (1 - beta) g + beta v, sign(v) packed into the send buffer."""
+        if self.momentum is not None:
+            self.B.ss_signum_update(grad, self.momentum, self.beta, self.ex.local_words(), stream)
+        else:
+            self.B.ss_sign_pack(grad, self.ex.local_words(), stream)
+
+    def serve(self, flip_mask: int = 0, stream=None) -> None:
+        """sharded mode: receive every worker's words of this worker's slice and vote on them
+        (this worker acting as the parameter server of its slice). No-op in allgather mode."""
+        ex = self.ex
+        if ex.mode != "sharded":
+            return
+        ex.scatter_slices()
+        n = ex.slice_coordinates()
+        if n > 0:
+            self.B.ss_majority_vote(ex.slice_rows(), n, flip_mask, ex.slice_vote(), stream)
+
+    def finish(self, flip_mask: int = 0, stream=None) -> torch.Tensor:
+        """Receive what the update needs (all packed vectors, or the voted slices), update the
+        parameters, and return the packed vote of the whole vector."""
+        B, ex = self.B, self.ex
+        if ex.mode == "allgather":
+            ex.gather()
+            B.ss_vote_apply(ex.worker_rows(), self.x, self.lr, self.weight_decay, flip_mask,
+                            self.vote, stream)
+            return self.vote
+        ex.gather_vote()
+        B.ss_apply_vote(self.x, ex.vote_words(), self.lr, self.weight_decay, stream)
+        return ex.vote_words()
+
+    def step(self, grad: torch.Tensor, flip_mask: int = 0, stream=None) -> torch.Tensor:
+        """One iteration. Kernels run on the current stream (or ``stream``, which must then be
+        the stream the collectives see as current)."""
+        self.pack_local(grad, stream)
+        self.serve(flip_mask, stream)
+        return self.finish(flip_mask, stream)

@@ -1,0 +1,103 @@
+"""MajorityVoteWorker on one GPU.
+
+Only one GPU is available to these tests, so the M workers of Algorithm 1 are M worker objects
+in one process whose collectives are served by an in-process stand-in that copies between their
+buffers (all on one stream, one after another: no kernel waits on another). The kernels, the
+buffers and the slice arithmetic are the ones a multi-GPU run uses; the NCCL transport itself is
+exercised with a one-rank process group. Every worker must end each step with the parameters,
+momentum and packed vote of the oracle's M-worker step.
+"""
+import os
+import socket
+
+import numpy as np
+import pytest
+import torch
+import torch.distributed as dist
+
+import oracle
+from paper_1810_05291_b200.distributed import MajorityVoteWorker
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+
+
+class InProcessFabric:
+    """Stand-in for torch.distributed inside one process: rank r's call is served at once from
+    the other ranks' buffers, which the test has filled in an earlier phase."""
+
+    def __init__(self):
+        self.workers = []
+
+    def endpoint(self, rank):
+        fabric = self
+
+        class Endpoint:
+            def all_gather_into_tensor(self, out, inp, group=None):
+                n = inp.numel()
+                for m, w in enumerate(fabric.workers):
+                    src = w.ex.local if inp is fabric.workers[rank].ex.local else w.ex.vote_slice
+                    out[m * n:(m + 1) * n].copy_(src)
+
+            def all_to_all_single(self, out, inp, group=None):
+                n = out.numel() // len(fabric.workers)
+                for m, w in enumerate(fabric.workers):
+                    out[m * n:(m + 1) * n].copy_(w.ex.local[rank * n:(rank + 1) * n])
+
+        return Endpoint()
+
+
+@pytest.mark.parametrize("mode", ["allgather", "sharded"])
+@pytest.mark.parametrize("M,d,beta,flip", [(3, 1000, None, 0), (7, 100_003, 0.9, 0b1000000),
+                                           (15, 32 * 3000 + 8, 0.9, 0), (4, 70, 0.9, 0b0011),
+                                           (5, 33, None, 0b00001)])
+def test_m_workers_in_one_process_match_the_oracle(M, d, beta, flip, mode):
+    rng = np.random.default_rng(100 * M + d)
+    x0 = rng.standard_normal(d).astype(np.float32)
+    fabric = InProcessFabric()
+    for m in range(M):
+        w = MajorityVoteWorker(torch.from_numpy(x0.copy()).to(DEV), beta, 1e-3, 0.01, mode,
+                               world=M, rank=m, collectives=fabric.endpoint(m))
+        fabric.workers.append(w)
+    ref_x = x0.copy()
+    ref_v = [np.zeros(d, dtype=np.float32) for _ in range(M)] if beta is not None else None
+    for step in range(3):
+        grads = [rng.standard_normal(d).astype(np.float32) for _ in range(M)]
+        want = oracle.fused_step(grads, ref_v, ref_x, beta if beta is not None else 0.0, 1e-3, 0.01, flip)
+        for m, w in enumerate(fabric.workers):
+            w.pack_local(torch.from_numpy(grads[m]).to(DEV))
+        for w in fabric.workers:
+            w.serve(flip)
+        votes = [w.finish(flip) for w in fabric.workers]
+        torch.cuda.synchronize()
+        for m, w in enumerate(fabric.workers):
+            assert np.array_equal(votes[m].cpu().numpy().view(np.uint32), want), "vote, worker %d" % m
+            assert np.array_equal(w.x.cpu().numpy().view(np.uint32), ref_x.view(np.uint32)), "x, worker %d" % m
+            if beta is not None:
+                assert np.array_equal(w.momentum.cpu().numpy().view(np.uint32), ref_v[m].view(np.uint32))
+
+
+@pytest.mark.parametrize("mode", ["allgather", "sharded"])
+def test_one_rank_nccl_group_runs_the_real_collectives(mode):
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        port = s.getsockname()[1]
+    os.environ["MASTER_ADDR"] = "127.0.0.1"
+    os.environ["MASTER_PORT"] = str(port)
+    torch.cuda.set_device(0)
+    dist.init_process_group("nccl", rank=0, world_size=1, device_id=torch.device(DEV))
+    try:
+        d = 32 * 5000 + 8
+        rng = np.random.default_rng(9)
+        x0 = rng.standard_normal(d).astype(np.float32)
+        w = MajorityVoteWorker(torch.from_numpy(x0.copy()).to(DEV), 0.9, 1e-3, 0.0, mode)
+        ref_x, ref_v = x0.copy(), [np.zeros(d, dtype=np.float32)]
+        for step in range(2):
+            g = rng.standard_normal(d).astype(np.float32)
+            want = oracle.fused_step([g], ref_v, ref_x, 0.9, 1e-3)
+            vote = w.step(torch.from_numpy(g).to(DEV))
+            torch.cuda.synchronize()
+            assert np.array_equal(vote.cpu().numpy().view(np.uint32), want)
+            assert np.array_equal(w.x.cpu().numpy().view(np.uint32), ref_x.view(np.uint32))
+    finally:
+        dist.destroy_process_group()
