@@ -102,6 +102,24 @@ int ss_signum_update(const void* grad, ss_dtype dt, float* momentum, float beta,
                      uint32_t* out_words, void* cuda_stream);
 
 /*
+ * ss_signum_update that also performs the first push of Algorithm 1 ("push sign(v_m) to
+ * server"): each packed word is stored to every one of n_dests buffers by the kernel that
+ * produces it. With one worker per GPU the destinations are the slot reserved for this worker
+ * in every worker's receive buffer -- its own and its peers', mapped into this process with
+ * peer access enabled -- so that the all-gather of packed words needs no separate collective.
+ * Only plain stores go to a peer; nothing is read from one. The caller orders the exchange:
+ * every worker's call must have completed (stream synchronisation plus a barrier across the
+ * workers) before any worker's ss_vote_apply reads its receive buffer, and the next step's push
+ * must not start before those reads have finished.
+ *   grad, momentum, beta, d   as ss_signum_update
+ *   dests    out  HOST array of n_dests device pointers, each to ceil(d/32) words, disjoint
+ *   n_dests  1 .. SS_MAX_WORKERS
+ * Every destination receives exactly what ss_signum_update would write.
+ */
+int ss_signum_update_push(const void* grad, ss_dtype dt, float* momentum, float beta, int64_t d,
+                          uint32_t* const* dests, int n_dests, void* cuda_stream);
+
+/*
  * Algorithm 1, "update parameters": x <- x - lr (sign(V) + weight_decay x) from the packed vote.
  *   param       in/out  d fp32
  *   vote_words  in      ceil(d/32) words

@@ -35,7 +35,7 @@ SS_ERR_CUDA = -4
 EXPORTS = ("ss_packed_words", "ss_status_string", "ss_last_cuda_error", "ss_sign_pack",
            "ss_majority_vote", "ss_signum_update", "ss_apply_vote", "ss_fused_step",
            "ss_segments_upload", "ss_fused_step_segments", "ss_apply_vote_segments",
-           "ss_vote_apply", "ss_vote_apply_segments", "ss_fused_step_host", "ss_fused_step_host_static", "ss_set_launch_option")
+           "ss_vote_apply", "ss_vote_apply_segments", "ss_signum_update_push", "ss_fused_step_host", "ss_fused_step_host_static", "ss_set_launch_option")
 
 
 class ss_segment(ctypes.Structure):
@@ -86,12 +86,14 @@ def lib() -> ctypes.CDLL:
     L.ss_segments_upload.argtypes = [vp, i32, i64, vp, vp]
     L.ss_fused_step_segments.argtypes = [vp, i32, vp, i32, i64, f32, u64, vp, vp, i32, vp, vp]
     L.ss_apply_vote_segments.argtypes = [vp, vp, i64, vp, i32, vp]
+    L.ss_signum_update_push.argtypes = [vp, i32, vp, f32, i64, vp, i32, vp]
     L.ss_vote_apply.argtypes = [vp, i32, i64, u64, vp, f32, f32, vp, vp]
     L.ss_vote_apply_segments.argtypes = [vp, i32, i64, u64, vp, vp, i32, vp, vp]
     for name in ("ss_sign_pack", "ss_majority_vote", "ss_signum_update", "ss_apply_vote",
                  "ss_fused_step", "ss_fused_step_host", "ss_fused_step_host_static",
                  "ss_set_launch_option", "ss_segments_upload", "ss_fused_step_segments",
-                 "ss_apply_vote_segments", "ss_vote_apply", "ss_vote_apply_segments"):
+                 "ss_apply_vote_segments", "ss_vote_apply", "ss_vote_apply_segments",
+                 "ss_signum_update_push"):
         getattr(L, name).restype = i32
     _lib = L
     return L
@@ -173,6 +175,17 @@ def ss_signum_update(grad: torch.Tensor, momentum: torch.Tensor, beta: float,
                                   _dev(momentum, torch.float32, "momentum", d), float(beta), d,
                                   _words(out_words, d, "out_words"), _stream(stream)),
            "ss_signum_update")
+
+
+def ss_signum_update_push(grad: torch.Tensor, momentum: torch.Tensor, beta: float,
+                          dests: Sequence[torch.Tensor], stream=None) -> None:
+    """``dests`` may be tensors on this GPU or raw integer addresses of peer buffers."""
+    d = grad.numel()
+    ptrs = [p if isinstance(p, int) else _words(p, d, "dests[%d]" % i) for i, p in enumerate(dests)]
+    _check(lib().ss_signum_update_push(_dev(grad, None, "grad"), _dtype_code(grad),
+                                       _dev(momentum, torch.float32, "momentum", d), float(beta), d,
+                                       _ptr_array(ptrs), len(ptrs), _stream(stream)),
+           "ss_signum_update_push")
 
 
 def ss_apply_vote(param: torch.Tensor, vote_words: torch.Tensor, lr: float,

@@ -160,6 +160,41 @@ int ss_signum_update(const void* grad, ss_dtype dt, float* momentum, float beta,
     return step_common(g, dt, v, 1, d, beta, 0, nullptr, 0.0f, 0.0f, out_words, cuda_stream);
 }
 
+int ss_signum_update_push(const void* grad, ss_dtype dt, float* momentum, float beta, int64_t d,
+                          uint32_t* const* dests, int n_dests, void* cuda_stream) {
+    if (!dtype_ok(dt) || d < 0 || n_dests < 1 || n_dests > SS_MAX_WORKERS) return SS_ERR_INVALID_ARG;
+    if (d == 0) return SS_OK;
+    if (grad == nullptr || momentum == nullptr || dests == nullptr) return SS_ERR_INVALID_ARG;
+    const size_t eb = static_cast<size_t>(elem_bytes(dt));
+    const size_t gbytes = static_cast<size_t>(d) * eb, fbytes = static_cast<size_t>(d) * 4;
+    const size_t wbytes = static_cast<size_t>((d + 31) / 32) * 4;
+    if (!aligned(grad, eb) || !aligned(momentum, 4)) return SS_ERR_MISALIGNED;
+    if (overlap(grad, gbytes, momentum, fbytes)) return SS_ERR_INVALID_ARG;
+    for (int p = 0; p < n_dests; ++p) {
+        if (dests[p] == nullptr) return SS_ERR_INVALID_ARG;
+        if (!aligned(dests[p], 4)) return SS_ERR_MISALIGNED;
+        if (overlap(dests[p], wbytes, momentum, fbytes) || overlap(dests[p], wbytes, grad, gbytes))
+            return SS_ERR_INVALID_ARG;
+        for (int q = 0; q < p; ++q)
+            if (overlap(dests[p], wbytes, dests[q], wbytes)) return SS_ERR_INVALID_ARG;
+    }
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    if (aligned(grad, eb * 4) && aligned(momentum, 16)) {
+        const float omb = 1.0f - beta;
+        return cuda_status(dt == SS_F32
+                               ? launch_signum_push_f32(grad, momentum, beta, omb, d, dests, n_dests, st)
+                               : launch_signum_push_bf16(grad, momentum, beta, omb, d, dests, n_dests, st));
+    }
+    // pointers off the 16-byte grid: the scalar-load kernel into the first destination, then copies
+    const int rc = ss_signum_update(grad, dt, momentum, beta, d, dests[0], cuda_stream);
+    if (rc != SS_OK) return rc;
+    for (int p = 1; p < n_dests; ++p) {
+        cudaError_t e = cudaMemcpyAsync(dests[p], dests[0], wbytes, cudaMemcpyDefault, st);
+        if (e != cudaSuccess) return cuda_status(e);
+    }
+    return SS_OK;
+}
+
 int ss_fused_step(const void* const* grads, ss_dtype dt, float* const* momenta, int M, int64_t d,
                   float beta, uint64_t flip_mask, float* param, float lr, float weight_decay,
                   uint32_t* vote_words_out, void* cuda_stream) {

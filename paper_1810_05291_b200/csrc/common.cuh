@@ -165,6 +165,10 @@ struct StepDesc {
 
 cudaError_t launch_step_f32(const StepDesc& s, cudaStream_t st);
 cudaError_t launch_step_bf16(const StepDesc& s, cudaStream_t st);
+cudaError_t launch_signum_push_f32(const void* g, float* v, float beta, float omb, int64_t d,
+                                   uint32_t* const* dests, int n, cudaStream_t st);
+cudaError_t launch_signum_push_bf16(const void* g, float* v, float beta, float omb, int64_t d,
+                                    uint32_t* const* dests, int n, cudaStream_t st);
 cudaError_t launch_vote(const uint32_t* const* packed, int M, int64_t d, uint64_t flip,
                         uint32_t* vote, bool vec, cudaStream_t st);
 cudaError_t launch_vote_apply(const uint32_t* const* packed, int M, int64_t d, uint64_t flip,

@@ -5,4 +5,8 @@
 
 namespace ss {
 cudaError_t launch_step_bf16(const StepDesc& s, cudaStream_t st) { return launch_step_dtype<BF16>(s, st); }
+cudaError_t launch_signum_push_bf16(const void* g, float* v, float beta, float omb, int64_t d,
+                                   uint32_t* const* dests, int n, cudaStream_t st) {
+    return launch_signum_push<BF16>(g, v, beta, omb, d, dests, n, st);
+}
 }  // namespace ss

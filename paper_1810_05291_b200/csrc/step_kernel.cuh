@@ -399,6 +399,80 @@ cudaError_t launch_pack(const StepDesc& s, cudaStream_t st) {
     return cudaGetLastError();
 }
 
+// ss_signum_update with the all-gather of the packed words folded into the producing kernel:
+// every word is stored to n destination buffers, which may be other GPUs' memory mapped into
+// this process (plain peer stores over NVLink; no multicast, nothing is read from a peer). The
+// words are 1/96 of the bytes this kernel moves, so the remote stores ride along with the
+// momentum pass instead of a separate collective reading the words back from HBM.
+struct PushDests {
+    uint32_t* p[SS_MAX_WORKERS];
+    int n;
+};
+
+template <typename GT, int U>
+__global__ void __launch_bounds__(256)
+signum_push_kernel(const void* __restrict__ g, float* __restrict__ v, float beta, float omb,
+                   int64_t d, const __grid_constant__ PushDests dst) {
+    const int lane = threadIdx.x & 31;
+    const int k = lane & 7;
+    const int64_t n_quads = (d >> 5) << 3;
+    const int64_t tile = static_cast<int64_t>(blockDim.x) * U;
+    for (int64_t base = static_cast<int64_t>(blockIdx.x) * tile; base < n_quads;
+         base += static_cast<int64_t>(gridDim.x) * tile) {
+        float4 gq[U], vq[U];
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const int64_t q = base + static_cast<int64_t>(u) * blockDim.x + threadIdx.x;
+            const bool ok = q < n_quads;
+            gq[u] = ok ? GT::load4(g, q) : make_float4(-1.f, -1.f, -1.f, -1.f);
+            vq[u] = ok ? __ldcs(reinterpret_cast<const float4*>(v) + q) : make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const int64_t q = base + static_cast<int64_t>(u) * blockDim.x + threadIdx.x;
+            const bool ok = q < n_quads;
+            const float4 s = momentum_rn4(omb, gq[u], beta, vq[u]);
+            if (ok) __stcs(reinterpret_cast<float4*>(v) + q, s);
+            uint32_t w = (ok ? sign_nibble(s) : 0u) << (4 * k);
+            w |= __shfl_xor_sync(0xFFFFFFFFu, w, 1);
+            w |= __shfl_xor_sync(0xFFFFFFFFu, w, 2);
+            w |= __shfl_xor_sync(0xFFFFFFFFu, w, 4);
+            if (k == 0 && ok)
+                for (int p = 0; p < dst.n; ++p) dst.p[p][q >> 3] = w;
+        }
+    }
+    if ((d & 31) != 0 && blockIdx.x == 0 && threadIdx.x < 32) {
+        const int64_t c = ((d >> 5) << 5) + lane;
+        float s = -1.0f;
+        if (c < d) {
+            s = momentum_rn(omb, GT::load1(g, c), beta, v[c]);
+            v[c] = s;
+        }
+        const uint32_t w = __ballot_sync(0xFFFFFFFFu, c < d && s >= 0.0f);
+        if (lane == 0)
+            for (int p = 0; p < dst.n; ++p) dst.p[p][d >> 5] = w;
+    }
+}
+
+template <typename GT>
+cudaError_t launch_signum_push(const void* g, float* v, float beta, float omb, int64_t d,
+                               uint32_t* const* dests, int n, cudaStream_t st) {
+    PushDests dst;
+    for (int p = 0; p < SS_MAX_WORKERS; ++p) dst.p[p] = p < n ? dests[p] : nullptr;
+    dst.n = n;
+    int threads = launch_options().threads > 0 ? launch_options().threads : 256;
+    if (threads > 256) threads = 256;
+    constexpr int U = 4;
+    auto kernel = signum_push_kernel<GT, U>;
+    const int64_t quads = (d >> 5) << 3;
+    const int64_t tile = static_cast<int64_t>(threads) * U;
+    int grid = 1;
+    cudaError_t err = pick_grid(kernel, threads, (quads + tile - 1) / tile, &grid);
+    if (err != cudaSuccess) return err;
+    kernel<<<grid, threads, 0, st>>>(g, v, beta, omb, d, dst);
+    return cudaGetLastError();
+}
+
 template <int M_CT, typename GT, bool MOM, bool APPLY, bool VEC, bool SEG = false>
 cudaError_t launch_step_inst(const StepDesc& s, cudaStream_t st) {
     using S = StepShape<M_CT, MOM>;

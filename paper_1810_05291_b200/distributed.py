@@ -14,6 +14,13 @@ this GPU's own memory before a kernel reads them.
                it (``ss_majority_vote``); an all-gather returns the voted slices, and
                ``ss_apply_vote`` updates the parameters: about 2 (M-1)/M d/8 bytes per worker.
 
+``push``       the all-gather folded into the producing kernel: ``ss_signum_update_push`` stores
+               each packed word straight into this worker's slot of every worker's receive
+               buffer (peer stores over NVLink), a barrier across the workers follows, and
+               ``ss_vote_apply`` reads the local receive buffer. The caller supplies the peer
+               addresses (``set_push_destinations``) and the barrier. Signum only. Not run on
+               more than one GPU here: on one GPU the destinations are local buffers.
+
 ``PackedExchange`` holds the buffers and the slice arithmetic and works on any device (the
 multi-process CPU tests drive it over gloo); ``MajorityVoteWorker`` adds the kernels and needs
 CUDA tensors. There is no CPU path for the arithmetic.
@@ -36,8 +43,8 @@ class PackedExchange:
 
     def __init__(self, d: int, world: int, rank: int, device, mode: str = "allgather", group=None,
                  collectives=None):
-        if mode not in ("allgather", "sharded"):
-            raise ValueError("mode must be 'allgather' or 'sharded'")
+        if mode not in ("allgather", "sharded", "push"):
+            raise ValueError("mode must be 'allgather', 'sharded' or 'push'")
         if world < 1 or not 0 <= rank < world or d < 0:
             raise ValueError("bad world/rank/d")
         self.d, self.world, self.rank, self.mode, self.group = int(d), world, rank, mode, group
@@ -47,7 +54,7 @@ class PackedExchange:
         self.W_pad = self.slice_words * world               # local buffer, padded with zero words
         kw = dict(dtype=torch.int32, device=device)
         self.local = torch.zeros(self.W_pad, **kw)          # this worker's packed sign(v)
-        if mode == "allgather":
+        if mode in ("allgather", "push"):
             self.gathered = torch.zeros(world * self.W_pad, **kw)
         else:
             self.recv = torch.zeros(world * self.slice_words, **kw)
@@ -62,6 +69,10 @@ class PackedExchange:
     def worker_rows(self) -> List[torch.Tensor]:
         """allgather mode, after gather(): worker m's packed vector, m = 0..M-1."""
         return [self.gathered[m * self.W_pad: m * self.W_pad + self.W] for m in range(self.world)]
+
+    def slot(self, m: int) -> torch.Tensor:
+        """push mode: the part of this worker's receive buffer that worker m writes."""
+        return self.gathered[m * self.W_pad: m * self.W_pad + self.W]
 
     def slice_coordinates(self) -> int:
         """sharded mode: how many of the d coordinates fall in this worker's server slice."""
@@ -93,7 +104,7 @@ class PackedExchange:
 
     def bytes_received_per_step(self) -> int:
         """Bytes this worker receives from its peers per iteration (excludes its own share)."""
-        if self.mode == "allgather":
+        if self.mode in ("allgather", "push"):
             return (self.world - 1) * self.W_pad * 4
         return 2 * (self.world - 1) * self.slice_words * 4
 
@@ -120,10 +131,28 @@ class MajorityVoteWorker:
         self.momentum = torch.zeros_like(param) if beta is not None else None
         self.ex = PackedExchange(self.d, world, rank, param.device, mode, group, collectives)
         self.vote = torch.zeros(self.ex.W, dtype=torch.int32, device=param.device)
+        self.push_dests = None
+        self.barrier = None
+        if mode == "push" and beta is None:
+            raise ValueError("push mode carries the momentum kernel: use it with Signum (beta set)")
+
+    def set_push_destinations(self, dests, barrier) -> None:
+        """push mode: ``dests[m]`` is the address (tensor or int) of this worker's slot in worker
+        m's receive buffer; ``barrier()`` must return only when every worker's push kernel has
+        completed, and is called again after the update so that no worker's next push overtakes
+        another worker's reads."""
+        if len(dests) != self.ex.world:
+            raise ValueError("need one destination per worker")
+        self.push_dests = list(dests)
+        self.barrier = barrier
 
     def pack_local(self, grad: torch.Tensor, stream=None) -> None:
         """Worker side: v <- (1 - beta) g + beta v, sign(v) packed into the send buffer."""
-        if self.momentum is not None:
+        if self.ex.mode == "push":
+            if self.push_dests is None:
+                raise RuntimeError("push mode: call set_push_destinations first")
+            self.B.ss_signum_update_push(grad, self.momentum, self.beta, self.push_dests, stream)
+        elif self.momentum is not None:
             self.B.ss_signum_update(grad, self.momentum, self.beta, self.ex.local_words(), stream)
         else:
             self.B.ss_sign_pack(grad, self.ex.local_words(), stream)
@@ -143,6 +172,12 @@ class MajorityVoteWorker:
         """Receive what the update needs (all packed vectors, or the voted slices), update the
         parameters, and return the packed vote of the whole vector."""
         B, ex = self.B, self.ex
+        if ex.mode == "push":
+            self.barrier()
+            B.ss_vote_apply(ex.worker_rows(), self.x, self.lr, self.weight_decay, flip_mask,
+                            self.vote, stream)
+            self.barrier()
+            return self.vote
         if ex.mode == "allgather":
             ex.gather()
             B.ss_vote_apply(ex.worker_rows(), self.x, self.lr, self.weight_decay, flip_mask,

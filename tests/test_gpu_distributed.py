@@ -77,6 +77,31 @@ def test_m_workers_in_one_process_match_the_oracle(M, d, beta, flip, mode):
                 assert np.array_equal(w.momentum.cpu().numpy().view(np.uint32), ref_v[m].view(np.uint32))
 
 
+@pytest.mark.parametrize("M,d,flip", [(3, 1000, 0), (7, 100_003, 0b0100000), (15, 32 * 3000 + 8, 0)])
+def test_push_mode_fills_every_workers_receive_buffer(M, d, flip):
+    rng = np.random.default_rng(7 * M + d)
+    x0 = rng.standard_normal(d).astype(np.float32)
+    workers = [MajorityVoteWorker(torch.from_numpy(x0.copy()).to(DEV), 0.9, 1e-3, 0.0, "push",
+                                  world=M, rank=m) for m in range(M)]
+    calls = []
+    for m, w in enumerate(workers):           # worker m's slot in every worker's receive buffer
+        w.set_push_destinations([peer.ex.slot(m) for peer in workers], lambda: calls.append(1))
+    ref_x = x0.copy()
+    ref_v = [np.zeros(d, dtype=np.float32) for _ in range(M)]
+    for step in range(3):
+        grads = [rng.standard_normal(d).astype(np.float32) for _ in range(M)]
+        want = oracle.fused_step(grads, ref_v, ref_x, 0.9, 1e-3, 0.0, flip)
+        for m, w in enumerate(workers):
+            w.pack_local(torch.from_numpy(grads[m]).to(DEV))
+        votes = [w.finish(flip) for w in workers]
+        torch.cuda.synchronize()
+        for m, w in enumerate(workers):
+            assert np.array_equal(votes[m].cpu().numpy().view(np.uint32), want)
+            assert np.array_equal(w.x.cpu().numpy().view(np.uint32), ref_x.view(np.uint32))
+            assert np.array_equal(w.momentum.cpu().numpy().view(np.uint32), ref_v[m].view(np.uint32))
+    assert len(calls) == 3 * M * 2
+
+
 @pytest.mark.parametrize("mode", ["allgather", "sharded"])
 def test_one_rank_nccl_group_runs_the_real_collectives(mode):
     with socket.socket() as s:

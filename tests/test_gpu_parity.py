@@ -116,6 +116,25 @@ def test_signum_update(d, misalign, dtype):
     check_guard(full, lo, d)
 
 
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16], ids=["f32", "bf16"])
+@pytest.mark.parametrize("misalign", [0, 1], ids=["aligned", "unaligned"])
+@pytest.mark.parametrize("n_dests", [1, 3, 8])
+@pytest.mark.parametrize("d", [1, 33, 4097, 100_003, 32 * 4096 + 8])
+def test_signum_update_push(d, n_dests, misalign, dtype):
+    g = _rand(d + misalign, 210 + d, dtype)[misalign:]
+    full, v, lo = guarded_f32(_rand(d, 310 + d, specials=False), misalign)
+    v_np, g_np = to_np(v), to_np(g)
+    outs = [GuardedWords(d, DEV) for _ in range(n_dests)]
+    for step in range(2):
+        B.ss_signum_update_push(g, v, 0.9, [o.view for o in outs])
+        want = oracle.signum_update(g_np, v_np, 0.9)
+        for o in outs:
+            assert_words_equal(o.view, want, "pushed words step %d" % step)
+            o.check()
+        assert count_bit_mismatch(v, v_np) == 0
+    check_guard(full, lo, d)
+
+
 @pytest.mark.parametrize("M", ALL_M)
 @pytest.mark.parametrize("misalign", [0, 1], ids=["aligned", "unaligned"])
 @pytest.mark.parametrize("d", [1, 33, 127, 128, 4097, 100_003])
