@@ -92,6 +92,18 @@ int ss_majority_vote(const uint32_t* const* packed, int M, int64_t d, uint64_t f
                      uint32_t* vote_words, void* cuda_stream);
 
 /*
+ * The tally of Algorithm 1's server line itself, V = sum_m sign(v_m), one int8 per coordinate
+ * (-M <= V <= M, same parity as M). A diagnostic, not a step of the iteration: it gives the
+ * margin of every vote (V = 2 Z - M with Z the count of +1 votes that the proof of Theorem 2
+ * bounds), e.g. to compare measured vote failures with that theorem's bound.
+ *   packed     in   HOST array of M device pointers, each to ceil(d/32) words
+ *   tally_out  out  d int8 (any alignment)
+ * sign of the tally under the header's sign rule (V >= 0 -> +1) is what ss_majority_vote packs.
+ */
+int ss_vote_tally(const uint32_t* const* packed, int M, int64_t d, uint64_t flip_mask,
+                  int8_t* tally_out, void* cuda_stream);
+
+/*
  * Worker side of Algorithm 1 with momentum: v <- (1 - beta) g + beta v in place, then sign(v)
  * packed. beta = 0 gives the packed sign of g (and v = g).
  *   grad       in      d elements of dtype dt

@@ -35,7 +35,7 @@ SS_ERR_CUDA = -4
 EXPORTS = ("ss_packed_words", "ss_status_string", "ss_last_cuda_error", "ss_sign_pack",
            "ss_majority_vote", "ss_signum_update", "ss_apply_vote", "ss_fused_step",
            "ss_segments_upload", "ss_fused_step_segments", "ss_apply_vote_segments",
-           "ss_vote_apply", "ss_vote_apply_segments", "ss_signum_update_push", "ss_fused_step_host", "ss_fused_step_host_static", "ss_set_launch_option")
+           "ss_vote_apply", "ss_vote_apply_segments", "ss_signum_update_push", "ss_vote_tally", "ss_fused_step_host", "ss_fused_step_host_static", "ss_set_launch_option")
 
 
 class ss_segment(ctypes.Structure):
@@ -87,13 +87,14 @@ def lib() -> ctypes.CDLL:
     L.ss_fused_step_segments.argtypes = [vp, i32, vp, i32, i64, f32, u64, vp, vp, i32, vp, vp]
     L.ss_apply_vote_segments.argtypes = [vp, vp, i64, vp, i32, vp]
     L.ss_signum_update_push.argtypes = [vp, i32, vp, f32, i64, vp, i32, vp]
+    L.ss_vote_tally.argtypes = [vp, i32, i64, u64, vp, vp]
     L.ss_vote_apply.argtypes = [vp, i32, i64, u64, vp, f32, f32, vp, vp]
     L.ss_vote_apply_segments.argtypes = [vp, i32, i64, u64, vp, vp, i32, vp, vp]
     for name in ("ss_sign_pack", "ss_majority_vote", "ss_signum_update", "ss_apply_vote",
                  "ss_fused_step", "ss_fused_step_host", "ss_fused_step_host_static",
                  "ss_set_launch_option", "ss_segments_upload", "ss_fused_step_segments",
                  "ss_apply_vote_segments", "ss_vote_apply", "ss_vote_apply_segments",
-                 "ss_signum_update_push"):
+                 "ss_signum_update_push", "ss_vote_tally"):
         getattr(L, name).restype = i32
     _lib = L
     return L
@@ -186,6 +187,14 @@ def ss_signum_update_push(grad: torch.Tensor, momentum: torch.Tensor, beta: floa
                                        _dev(momentum, torch.float32, "momentum", d), float(beta), d,
                                        _ptr_array(ptrs), len(ptrs), _stream(stream)),
            "ss_signum_update_push")
+
+
+def ss_vote_tally(packed: Sequence[torch.Tensor], d: int, flip_mask: int, tally_out: torch.Tensor,
+                  stream=None) -> None:
+    ptrs = [_words(p, d, "packed[%d]" % m) for m, p in enumerate(packed)]
+    _check(lib().ss_vote_tally(_ptr_array(ptrs), len(ptrs), int(d), int(flip_mask),
+                               _dev(tally_out, torch.int8, "tally_out", int(d)), _stream(stream)),
+           "ss_vote_tally")
 
 
 def ss_apply_vote(param: torch.Tensor, vote_words: torch.Tensor, lr: float,

@@ -227,6 +227,22 @@ int ss_majority_vote(const uint32_t* const* packed, int M, int64_t d, uint64_t f
                                    static_cast<cudaStream_t>(cuda_stream)));
 }
 
+int ss_vote_tally(const uint32_t* const* packed, int M, int64_t d, uint64_t flip_mask,
+                  int8_t* tally_out, void* cuda_stream) {
+    if (packed == nullptr || M < 1 || M > SS_MAX_WORKERS || d < 0) return SS_ERR_INVALID_ARG;
+    if (!flip_ok(flip_mask, M)) return SS_ERR_INVALID_ARG;
+    if (d == 0) return SS_OK;
+    if (tally_out == nullptr) return SS_ERR_INVALID_ARG;
+    const size_t wbytes = static_cast<size_t>((d + 31) / 32) * 4;
+    for (int m = 0; m < M; ++m) {
+        if (packed[m] == nullptr) return SS_ERR_INVALID_ARG;
+        if (!aligned(packed[m], 4)) return SS_ERR_MISALIGNED;
+        if (overlap(packed[m], wbytes, tally_out, static_cast<size_t>(d))) return SS_ERR_INVALID_ARG;
+    }
+    return cuda_status(launch_tally(packed, M, d, flip_mask, tally_out,
+                                    static_cast<cudaStream_t>(cuda_stream)));
+}
+
 int ss_apply_vote(float* param, const uint32_t* vote_words, int64_t d, float lr, float weight_decay,
                   void* cuda_stream) {
     if (d < 0) return SS_ERR_INVALID_ARG;

@@ -174,6 +174,8 @@ cudaError_t launch_vote(const uint32_t* const* packed, int M, int64_t d, uint64_
 cudaError_t launch_vote_apply(const uint32_t* const* packed, int M, int64_t d, uint64_t flip,
                               float* x, float lr, float wd, bool vec, const ss_segment* seg,
                               int n_seg, uint32_t* vote, cudaStream_t st);
+cudaError_t launch_tally(const uint32_t* const* packed, int M, int64_t d, uint64_t flip, int8_t* out,
+                         cudaStream_t st);
 cudaError_t launch_apply(float* x, const uint32_t* vote, int64_t d, float lr, float wd, bool vec,
                          const ss_segment* seg, int n_seg, cudaStream_t st);
 

@@ -347,6 +347,121 @@ cudaError_t launch_vote_apply(const uint32_t* const* packed, int M, int64_t d, u
                : launch_vote_apply_m<false, false>(packed, M, d, flip, x, lr, wd, seg, n_seg, vote, st);
 }
 
+// ---- the tally itself: V = sum_m sign(v_m) per coordinate as int8 (a diagnostic: the margin by
+// which each vote was won, the quantity Z of Theorem 2's proof). A warp owns 32 words: lane l
+// counts word l of every worker bit-sliced, then in eight rounds each lane fetches the count
+// planes of the word that holds its four coordinates by shuffle, rebuilds the four counts and
+// stores four int8 at once (128 contiguous bytes per warp and round). -----------------------------
+
+template <int NP>
+struct TallyArgs {
+    const uint32_t* p[NP];
+    int8_t* out;
+    int64_t d;
+    uint64_t flip;
+    int M;
+    int out_aligned4;
+};
+
+template <int M_CT>
+__global__ void __launch_bounds__(256)
+vote_tally_kernel(const __grid_constant__ TallyArgs<VoteShape<M_CT>::NP> a) {
+    using S = VoteShape<M_CT>;
+    constexpr int LB = S::LB, P = S::P;
+    const int M = M_CT > 0 ? M_CT : a.M;
+    const int lane = threadIdx.x & 31;
+    const int64_t W = (a.d + 31) >> 5;
+    const int64_t n_tiles = (W + 31) >> 5;
+    const int64_t warps = (static_cast<int64_t>(gridDim.x) * blockDim.x) >> 5;
+    for (int64_t t = (static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x) >> 5; t < n_tiles;
+         t += warps) {
+        const int64_t j = (t << 5) + lane;
+        const bool jv = j < W;
+        BitCounter<P> cnt;
+        cnt.clear();
+        auto batch = [&](int m0, auto nb_tag) {
+            constexpr int NB = decltype(nb_tag)::value;
+            uint32_t w[NB];
+#pragma unroll
+            for (int k = 0; k < NB; ++k) {
+                const bool live = jv && (M_CT > 0 || m0 + k < M);
+                const int mi = m0 + k < S::NP ? m0 + k : 0;
+                w[k] = live ? __ldcs(a.p[mi] + j) : 0u;
+            }
+#pragma unroll
+            for (int k = 0; k < NB; ++k) {
+                const bool live = jv && (M_CT > 0 || m0 + k < M);
+                if (live && ((a.flip >> (m0 + k)) & 1ull)) w[k] = ~w[k];
+            }
+            cnt.template add_words<NB>(w);
+        };
+        if constexpr (M_CT > 0) {
+            constexpr int FULL = M_CT / LB, REM = M_CT % LB;
+#pragma unroll
+            for (int b = 0; b < FULL; ++b) batch(b * LB, std::integral_constant<int, LB>{});
+            if constexpr (REM > 0) batch(FULL * LB, std::integral_constant<int, REM>{});
+        } else {
+            for (int m0 = 0; m0 < M; m0 += LB) batch(m0, std::integral_constant<int, LB>{});
+        }
+#pragma unroll
+        for (int it = 0; it < 8; ++it) {
+            const int src = 4 * it + (lane >> 3);
+            uint32_t pl[P];
+#pragma unroll
+            for (int q = 0; q < P; ++q) pl[q] = __shfl_sync(0xFFFFFFFFu, cnt.p[q], src);
+            const int64_t c0 = (((t << 5) + src) << 5) + 4 * (lane & 7);
+            uint32_t four = 0u;
+#pragma unroll
+            for (int b = 0; b < 4; ++b) {
+                const int pos = 4 * (lane & 7) + b;
+                int count = 0;
+#pragma unroll
+                for (int q = 0; q < P; ++q) count |= static_cast<int>((pl[q] >> pos) & 1u) << q;
+                const int V = 2 * count - M;
+                four |= (static_cast<uint32_t>(V) & 0xFFu) << (8 * b);
+            }
+            if (c0 + 3 < a.d && a.out_aligned4) {
+                *reinterpret_cast<uint32_t*>(a.out + c0) = four;
+            } else {
+                for (int b = 0; b < 4; ++b)
+                    if (c0 + b < a.d) a.out[c0 + b] = static_cast<int8_t>((four >> (8 * b)) & 0xFFu);
+            }
+        }
+    }
+}
+
+template <int M_CT>
+cudaError_t launch_tally_inst(const uint32_t* const* packed, int M, int64_t d, uint64_t flip,
+                              int8_t* out, cudaStream_t st) {
+    using S = VoteShape<M_CT>;
+    TallyArgs<S::NP> a;
+    for (int m = 0; m < S::NP; ++m) a.p[m] = m < M ? packed[m] : nullptr;
+    a.out = out;
+    a.d = d;
+    a.flip = flip;
+    a.M = M;
+    a.out_aligned4 = (reinterpret_cast<uintptr_t>(out) & 3) == 0;
+    int threads = launch_options().threads > 0 ? launch_options().threads : 256;
+    if (threads > 256) threads = 256;
+    const int64_t tiles = (((d + 31) >> 5) + 31) >> 5;
+    const int64_t per_block = threads / 32;
+    int grid = 1;
+    auto kernel = vote_tally_kernel<M_CT>;
+    cudaError_t err = pick_grid(kernel, threads, (tiles + per_block - 1) / per_block, &grid);
+    if (err != cudaSuccess) return err;
+    kernel<<<grid, threads, 0, st>>>(a);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_tally(const uint32_t* const* packed, int M, int64_t d, uint64_t flip, int8_t* out,
+                         cudaStream_t st) {
+    switch (M) {
+        case 7: return launch_tally_inst<7>(packed, M, d, flip, out, st);
+        case 15: return launch_tally_inst<15>(packed, M, d, flip, out, st);
+        default: return launch_tally_inst<0>(packed, M, d, flip, out, st);
+    }
+}
+
 // ---- apply: x <- x - lr (sign(V) + wd x) from packed vote words ------------------------------
 
 struct ApplyArgs {

@@ -151,6 +151,30 @@ def test_majority_vote(d, misalign, M):
         out.check()
 
 
+@pytest.mark.parametrize("M", ALL_M)
+@pytest.mark.parametrize("misalign", [0, 1], ids=["aligned", "unaligned"])
+@pytest.mark.parametrize("d", [1, 3, 33, 127, 1023, 1027, 4097, 100_003])
+def test_vote_tally(d, misalign, M):
+    W = B.ss_packed_words(d)
+    gen = torch.Generator(device=DEV).manual_seed(29 * d + M)
+    packed = [torch.randint(-(1 << 31), 1 << 31, (W,), generator=gen, device=DEV,
+                            dtype=torch.int64).to(torch.int32) for _ in range(M)]
+    flip = int(torch.randint(0, 1 << 30, (1,), generator=gen, device=DEV).item()) & ((1 << M) - 1)
+    pad = 64
+    full = torch.full((d + 2 * pad + misalign,), 99, dtype=torch.int8, device=DEV)
+    out = full[pad + misalign: pad + misalign + d]
+    for f in (0, flip):
+        B.ss_vote_tally(packed, d, f, out)
+        vote, tally = oracle.majority_vote([to_np(p) for p in packed], d, f, return_tally=True)
+        got = out.cpu().numpy().astype(np.int32)
+        assert np.array_equal(got, tally)
+        assert bool((full[: pad + misalign] == 99).all()) and bool((full[pad + misalign + d:] == 99).all())
+        # the packed vote is the sign of the tally
+        words = words_tensor(d, DEV, fill=-1)
+        B.ss_majority_vote(packed, d, f, words)
+        assert_words_equal(words, oracle.sign_pack(tally.astype(np.float32)))
+
+
 @pytest.mark.parametrize("wd", [0.0, 0.01])
 @pytest.mark.parametrize("misalign", [0, 1], ids=["aligned", "unaligned"])
 @pytest.mark.parametrize("d", AWKWARD_D)
