@@ -255,7 +255,7 @@ def entry_bytes(case, entry: str) -> int:
         return 8 * d + wb
     if entry == "vote_apply":
         return M * wb + 8 * d
-    if entry == "fused":
+    if entry in ("fused", "fused_segments"):
         return algorithmic_bytes(case)
     if entry == "chain":
         per_worker = entry_bytes(case, "signum_update" if mom else "pack")
@@ -314,13 +314,15 @@ def table_mode(args) -> None:
     peak, peak_src = measured_peak()
     if args.table == "named":
         names = ["cfg1", "cfg2", "cfg3", "cfg4", "cfg4tie"]
-        entries = ["pack", "signum_update", "vote", "apply", "vote_apply", "chain", "chain_va", "fused"]
+        entries = ["pack", "signum_update", "vote", "apply", "vote_apply", "chain", "chain_va", "fused",
+                   "fused_segments"]
     elif args.table == "sweep":
         names = ["sweep:%d:%d" % (d, M) for d in inputs.SWEEP_D for M in inputs.SWEEP_M]
         entries = ["vote", "fused"]
     else:
         names = args.table.split(",")
-        entries = ["pack", "signum_update", "vote", "apply", "vote_apply", "chain", "chain_va", "fused"]
+        entries = ["pack", "signum_update", "vote", "apply", "vote_apply", "chain", "chain_va", "fused",
+                   "fused_segments"]
     rows = []
     for name in names:
         case = make_case(name, args.d)
@@ -335,6 +337,13 @@ def table_mode(args) -> None:
         for m in range(case.M):
             B.ss_sign_pack(grads[m], packed[m], stream)
         turn = [0]
+        # a fused flat vector of 161 tensors (the number of parameter tensors of ResNet-50) at
+        # seeded cut points, all with the workload's own lr and weight decay
+        n_seg = 161
+        cuts = torch.randint(1, max(2, case.d), (n_seg - 1,), generator=torch.Generator().manual_seed(5)).sort().values
+        seg_begins = [0] + [int(c) for c in cuts]
+        seg_table = B.segment_table(n_seg, dev)
+        B.ss_segments_upload(seg_begins, [case.lr] * n_seg, [case.weight_decay] * n_seg, case.d, seg_table, stream)
 
         def call(entry):
             m = turn[0] % case.M
@@ -350,6 +359,8 @@ def table_mode(args) -> None:
             elif entry == "fused":
                 B.ss_fused_step(grads, moms, x, beta, case.lr, case.weight_decay, case.flip_mask,
                                 vote, stream)
+            elif entry == "fused_segments":
+                B.ss_fused_step_segments(grads, moms, x, beta, seg_table, n_seg, case.flip_mask, vote, stream)
             elif entry == "vote_apply":
                 B.ss_vote_apply(packed, x, case.lr, case.weight_decay, case.flip_mask, None, stream)
             elif entry == "chain_va":

@@ -79,8 +79,10 @@ def run_case(case, steps: int, stats: bool = False, check_chain: bool = True):
           for a, b in wins]
     if check_chain:
         x_u = x.clone()
+        x_va = x.clone()
         moms_u = [v.clone() for v in moms] if moms is not None else None
         vote_u = words_tensor(d, DEV, fill=-1)
+        vote_va = words_tensor(d, DEV, fill=-1)
     result = {}
     for step in range(steps):
         s = inputs.signal(case, DEV, step)
@@ -106,6 +108,10 @@ def run_case(case, steps: int, stats: bool = False, check_chain: bool = True):
             packed = unfused_chain(case, grads, moms_u, x_u, vote_u)
             assert torch.equal(vote, vote_u), "fused and unfused vote differ at step %d" % step
             assert torch.equal(x.view(torch.int32), x_u.view(torch.int32))
+            # the same packed words through the one-pass vote + update
+            B.ss_vote_apply(packed, x_va, case.lr, case.weight_decay, case.flip_mask, vote_va)
+            assert torch.equal(vote, vote_va), "ss_vote_apply vote differs at step %d" % step
+            assert torch.equal(x.view(torch.int32), x_va.view(torch.int32))
             if moms is not None:
                 for a_, b_ in zip(moms, moms_u):
                     assert torch.equal(a_.view(torch.int32), b_.view(torch.int32))
@@ -262,3 +268,75 @@ def test_cfg5_sweep_largest_d_on_windows(M):
     # vote is balanced instead: each bit is +1 with probability 1/2 for odd M
     share = float(unpack_bits(vote, d).float().mean().item())
     assert abs(share - 0.5) < 5e-4
+
+
+def _window_table(begins, lrs, wds, a, b, d):
+    """The segment table restricted to coordinates [a, b), with begins relative to a."""
+    out_b, out_lr, out_wd = [], [], []
+    n = len(begins)
+    for k in range(n):
+        lo, hi = begins[k], begins[k + 1] if k + 1 < n else d
+        if hi > a and lo < b and hi > lo:
+            out_b.append(max(lo, a) - a)
+            out_lr.append(lrs[k])
+            out_wd.append(wds[k])
+    return out_b, out_lr, out_wd
+
+
+def test_cfg3_as_a_fused_vector_of_161_tensors():
+    """Tensor fusion at full size: the ResNet-50-sized vector cut into 161 tensors (that model's
+    number of parameter tensors) at seeded, unaligned coordinates, each with its own learning rate
+    and weight decay, against one oracle step per tensor on sampled windows."""
+    case = inputs.cfg3()
+    d, M, n_seg = case.d, case.M, 161
+    rng = np.random.default_rng(161)
+    begins = [0] + sorted(int(c) for c in rng.integers(1, d, size=n_seg - 1))
+    lrs = [float(10.0 ** rng.uniform(-5, -3)) for _ in range(n_seg)]
+    wds = [0.0 if k % 2 else float(10.0 ** rng.uniform(-4, -2)) for k in range(n_seg)]
+    tab = B.segment_table(n_seg, DEV)
+    B.ss_segments_upload(begins, lrs, wds, d, tab)
+    x = inputs.initial_params(case, DEV)
+    moms = inputs.zero_momenta(case, DEV)
+    vote = words_tensor(d, DEV, fill=-1)
+    # windows: the standard ones plus one around each of three tensor boundaries
+    wins = windows(d, seed=161)
+    for k in (1, 80, 160):
+        a = max(0, (begins[k] - 5000) // 32 * 32)
+        wins.append((a, min(d, a + 10_016)))
+    ox = [to_np(x[a:b]) for a, b in wins]
+    om = [[np.zeros(b - a, dtype=np.float32) for _ in range(M)] for a, b in wins]
+    for step in range(2):
+        s = inputs.signal(case, DEV, step)
+        grads = [inputs.worker_gradient(case, m, DEV, step, s) for m in range(M)]
+        B.ss_fused_step_segments(grads, moms, x, case.beta, tab, n_seg, 0, vote)
+        torch.cuda.synchronize()
+        for wi, (a, b) in enumerate(wins):
+            wb, wl, ww = _window_table(begins, lrs, wds, a, b, d)
+            want = oracle.fused_step_segments([to_np(g[a:b]) for g in grads], om[wi], ox[wi], case.beta,
+                                              wb, wl, ww)
+            if b - a >= 32 and a % 32 == 0 and (b % 32 == 0 or b == d):
+                assert_words_equal(vote[a // 32:(b + 31) // 32], want, "vote, window %d" % wi)
+            assert count_bit_mismatch(x[a:b], ox[wi]) == 0, "parameters, window %d, step %d" % (wi, step)
+            for m in range(M):
+                assert count_bit_mismatch(moms[m][a:b], om[wi][m]) == 0
+        del grads, s
+
+
+def test_cfg2_tally_margins_match_the_oracle_and_the_vote():
+    case = inputs.cfg2()
+    d, M = case.d, case.M
+    grads = inputs.gradients(case, DEV, 0)
+    packed = [words_tensor(d, DEV) for _ in range(M)]
+    for m in range(M):
+        B.ss_sign_pack(grads[m], packed[m])
+    del grads
+    tally = torch.full((d,), 99, dtype=torch.int8, device=DEV)
+    vote = words_tensor(d, DEV, fill=-1)
+    B.ss_vote_tally(packed, d, case.flip_mask, tally)
+    B.ss_majority_vote(packed, d, case.flip_mask, vote)
+    assert torch.equal(tally >= 0, unpack_bits(vote, d))           # the vote is the tally's sign
+    assert bool(((tally.int() + M) % 2 == 0).all()) and int(tally.abs().max()) <= M
+    for a, b in windows(d, n_random=3, seed=2):
+        _, want = oracle.majority_vote([to_np(p[a // 32:(b + 31) // 32]) for p in packed], b - a,
+                                       case.flip_mask, return_tally=True)
+        assert np.array_equal(tally[a:b].cpu().numpy().astype(np.int32), want)
