@@ -340,3 +340,38 @@ def test_cfg2_tally_margins_match_the_oracle_and_the_vote():
         _, want = oracle.majority_vote([to_np(p[a // 32:(b + 31) // 32]) for p in packed], b - a,
                                        case.flip_mask, return_tally=True)
         assert np.array_equal(tally[a:b].cpu().numpy().astype(np.int32), want)
+
+
+@pytest.mark.parametrize("M,momentum", [(1, False), (3, True)])
+def test_more_than_two_to_the_31_coordinates(M, momentum):
+    """A single vector longer than 2^31 coordinates (64-bit indexing inside one buffer), ragged
+    end included, on windows at the start, across the 2^31 and 2^32-byte marks, and at the end."""
+    d = (1 << 31) + 100_000 + 8
+    need = (M * (2 if momentum else 1) + 1) * d * 4 * 1.1
+    free, _ = torch.cuda.mem_get_info()
+    if free < need:
+        pytest.skip("not enough free device memory")
+    gen = torch.Generator(device=DEV).manual_seed(31)
+    grads = [torch.randn(d, generator=gen, device=DEV) for _ in range(M)]
+    x = torch.randn(d, generator=gen, device=DEV)
+    moms = [torch.randn(d, generator=gen, device=DEV) * 0.1 for _ in range(M)] if momentum else None
+    wins = [(0, 1 << 16), ((1 << 30) - 4096, (1 << 30) + 4096), ((1 << 31) - 4096, (1 << 31) + 4096),
+            (d - 70_000 - 8 - (d - 70_000 - 8) % 32, d)]
+    ox = [to_np(x[a:b]) for a, b in wins]
+    om = [[to_np(v[a:b]) for v in moms] if momentum else None for a, b in wins]
+    vote = words_tensor(d, DEV, fill=-1)
+    B.ss_fused_step(grads, moms, x, 0.9, 1e-3, 0.0, 0, vote)
+    packed = [words_tensor(d, DEV, fill=-1) for _ in range(M)]
+    for m in range(M):
+        B.ss_sign_pack(grads[m], packed[m])
+    torch.cuda.synchronize()
+    for wi, (a, b) in enumerate(wins):
+        g_np = [to_np(g[a:b]) for g in grads]
+        want = oracle.fused_step(g_np, om[wi], ox[wi], 0.9, 1e-3)
+        assert_words_equal(vote[a // 32:(b + 31) // 32], want, "vote words, window %d" % wi)
+        assert count_bit_mismatch(x[a:b], ox[wi]) == 0
+        if momentum:
+            for m in range(M):
+                assert count_bit_mismatch(moms[m][a:b], om[wi][m]) == 0
+        assert_words_equal(packed[0][a // 32:(b + 31) // 32], oracle.sign_pack(g_np[0]), "pack, window %d" % wi)
+    assert int(vote[-1].item()) & 0xFFFFFFFF & ~((1 << (d % 32)) - 1) == 0
