@@ -260,7 +260,7 @@ def entry_bytes(case, entry: str) -> int:
     if entry == "chain":
         per_worker = entry_bytes(case, "signum_update" if mom else "pack")
         return M * per_worker + entry_bytes(case, "vote") + entry_bytes(case, "apply")
-    if entry == "chain_va":
+    if entry in ("chain_va", "chain_va_graph"):
         per_worker = entry_bytes(case, "signum_update" if mom else "pack")
         return M * per_worker + entry_bytes(case, "vote_apply")
     raise ValueError(entry)
@@ -314,15 +314,15 @@ def table_mode(args) -> None:
     peak, peak_src = measured_peak()
     if args.table == "named":
         names = ["cfg1", "cfg2", "cfg3", "cfg4", "cfg4tie"]
-        entries = ["pack", "signum_update", "vote", "apply", "vote_apply", "chain", "chain_va", "fused",
-                   "fused_segments"]
+        entries = ["pack", "signum_update", "vote", "apply", "vote_apply", "chain", "chain_va",
+                   "chain_va_graph", "fused", "fused_segments"]
     elif args.table == "sweep":
         names = ["sweep:%d:%d" % (d, M) for d in inputs.SWEEP_D for M in inputs.SWEEP_M]
         entries = ["vote", "fused"]
     else:
         names = args.table.split(",")
-        entries = ["pack", "signum_update", "vote", "apply", "vote_apply", "chain", "chain_va", "fused",
-                   "fused_segments"]
+        entries = ["pack", "signum_update", "vote", "apply", "vote_apply", "chain", "chain_va",
+                   "chain_va_graph", "fused", "fused_segments"]
     rows = []
     for name in names:
         case = make_case(name, args.d)
@@ -370,6 +370,8 @@ def table_mode(args) -> None:
                     else:
                         B.ss_sign_pack(grads[k], packed[k], stream)
                 B.ss_vote_apply(packed, x, case.lr, case.weight_decay, case.flip_mask, None, stream)
+            elif entry == "chain_va_graph":
+                graph.replay()
             elif entry == "chain":
                 for k in range(case.M):
                     if mom:
@@ -378,6 +380,23 @@ def table_mode(args) -> None:
                         B.ss_sign_pack(grads[k], packed[k], stream)
                 B.ss_majority_vote(packed, case.d, case.flip_mask, vote, stream)
                 B.ss_apply_vote(x, vote, case.lr, case.weight_decay, stream)
+
+        # the unfused chain recorded once into a CUDA graph (one submission per iteration)
+        graph = None
+        if "chain_va_graph" in entries:
+            side = torch.cuda.Stream()
+            side.wait_stream(stream)
+            graph = torch.cuda.CUDAGraph()
+            with torch.cuda.stream(side):
+                with torch.cuda.graph(graph, stream=side):
+                    cs = torch.cuda.current_stream()
+                    for k in range(case.M):
+                        if mom:
+                            B.ss_signum_update(grads[k], moms[k], beta, packed[k], cs)
+                        else:
+                            B.ss_sign_pack(grads[k], packed[k], cs)
+                    B.ss_vote_apply(packed, x, case.lr, case.weight_decay, case.flip_mask, None, cs)
+            stream.wait_stream(side)
 
         for entry in entries:
             if entry == "signum_update" and not mom:

@@ -392,3 +392,40 @@ def test_host_entry_point_matches_device_entry_point():
     assert torch.equal(x1, x2)
     for a, b in zip(m1, m2):
         assert torch.equal(a, b)
+
+
+def test_unfused_chain_replays_from_a_cuda_graph():
+    """The kernels only enqueue work on the caller's stream, so a whole iteration of the unfused
+    chain can be recorded once into a CUDA graph and replayed; the replays must give what the
+    same calls give when issued one by one."""
+    M, d = 7, 32 * 20_000 + 8
+    grads = [_rand(d, 8000 + m, specials=False) for m in range(M)]
+    x_e = _rand(d, 8100, specials=False)
+    x_g = x_e.clone()
+    mom_e = [torch.zeros(d, device=DEV) for _ in range(M)]
+    mom_g = [torch.zeros(d, device=DEV) for _ in range(M)]
+    packed = [words_tensor(d, DEV) for _ in range(M)]
+    vote_e, vote_g = words_tensor(d, DEV), words_tensor(d, DEV)
+
+    def chain(moms, x, vote):
+        for m in range(M):
+            B.ss_signum_update(grads[m], moms[m], 0.9, packed[m])
+        B.ss_vote_apply(packed, x, 1e-3, 0.0, 0b10, vote)
+
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(side):
+        with torch.cuda.graph(graph, stream=side):
+            chain(mom_g, x_g, vote_g)
+    torch.cuda.current_stream().wait_stream(side)
+    # capture does not run the work: the graph's buffers are still untouched
+    assert torch.equal(x_g, x_e)
+    for step in range(3):
+        graph.replay()
+        chain(mom_e, x_e, vote_e)
+        torch.cuda.synchronize()
+        assert torch.equal(vote_g, vote_e)
+        assert torch.equal(x_g.view(torch.int32), x_e.view(torch.int32))
+        for a, b in zip(mom_g, mom_e):
+            assert torch.equal(a.view(torch.int32), b.view(torch.int32))
