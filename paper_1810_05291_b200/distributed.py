@@ -146,6 +146,27 @@ class MajorityVoteWorker:
         self.push_dests = list(dests)
         self.barrier = barrier
 
+    def connect_push(self, group=None) -> None:
+        """push mode across GPUs: allocates the receive buffer in symmetric memory
+        (``torch.distributed._symmetric_memory``), exchanges its addresses over ``group``, and
+        points this worker's push at its own slot in every peer's buffer. The barrier is the
+        handle's stream-ordered barrier, so push kernel, barrier, vote + update and second barrier
+        run in order on the current stream without host synchronisation. Every worker of the
+        group must call this once, after the process group exists."""
+        import torch.distributed._symmetric_memory as symm
+        if self.ex.mode != "push":
+            raise RuntimeError("connect_push is for push mode")
+        group = group if group is not None else dist.group.WORLD
+        ex = self.ex
+        buf = symm.empty(ex.world * ex.W_pad, dtype=torch.int32, device=self.x.device)
+        buf.zero_()
+        handle = symm.rendezvous(buf, group)
+        ex.gathered = buf
+        slot_bytes = ex.W_pad * 4
+        dests = [int(handle.buffer_ptrs[m]) + ex.rank * slot_bytes for m in range(ex.world)]
+        self._symmetric = (buf, handle)
+        self.set_push_destinations(dests, handle.barrier)
+
     def pack_local(self, grad: torch.Tensor, stream=None) -> None:
         """Worker side: v <- (1 - beta) g + beta v, sign(v) packed into the send buffer."""
         if self.ex.mode == "push":

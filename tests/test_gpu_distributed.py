@@ -126,3 +126,35 @@ def test_one_rank_nccl_group_runs_the_real_collectives(mode):
             assert np.array_equal(w.x.cpu().numpy().view(np.uint32), ref_x.view(np.uint32))
     finally:
         dist.destroy_process_group()
+
+
+def test_push_mode_over_symmetric_memory_with_one_rank():
+    """The symmetric-memory wiring of push mode on a one-rank group: the receive buffer is a
+    symmetric allocation, the push goes to the address the rendezvous reports, and the handle's
+    barrier orders the steps. (More ranks need more GPUs than these tests have.)"""
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        port = s.getsockname()[1]
+    os.environ["MASTER_ADDR"] = "127.0.0.1"
+    os.environ["MASTER_PORT"] = str(port)
+    torch.cuda.set_device(0)
+    dist.init_process_group("nccl", rank=0, world_size=1, device_id=torch.device(DEV))
+    try:
+        d = 32 * 5000 + 8
+        rng = np.random.default_rng(19)
+        x0 = rng.standard_normal(d).astype(np.float32)
+        w = MajorityVoteWorker(torch.from_numpy(x0.copy()).to(DEV), 0.9, 1e-3, 0.0, "push")
+        try:
+            w.connect_push()
+        except (RuntimeError, NotImplementedError) as e:
+            pytest.skip("symmetric memory is not available here: %s" % str(e)[:200])
+        ref_x, ref_v = x0.copy(), [np.zeros(d, dtype=np.float32)]
+        for step in range(3):
+            g = rng.standard_normal(d).astype(np.float32)
+            want = oracle.fused_step([g], ref_v, ref_x, 0.9, 1e-3)
+            vote = w.step(torch.from_numpy(g).to(DEV))
+            torch.cuda.synchronize()
+            assert np.array_equal(vote.cpu().numpy().view(np.uint32), want)
+            assert np.array_equal(w.x.cpu().numpy().view(np.uint32), ref_x.view(np.uint32))
+    finally:
+        dist.destroy_process_group()
