@@ -34,7 +34,7 @@ NOMINAL_HBM_GBS = 8000.0
 # coordinate is touched exactly once). Keyed by (M, gradient bytes, momentum). An entry is
 # removed when its kernel changes until the counters are taken again.
 NCU_DRAM_BYTES_PER_COORD = {
-    (15, 4, True): (1.040216e9 + 487.84e6) / 8388608,
+    (15, 4, True): (1.040227e9 + 489.57e6) / 8388608,
 }
 
 
