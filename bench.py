@@ -35,6 +35,7 @@ NOMINAL_HBM_GBS = 8000.0
 # removed when its kernel changes until the counters are taken again.
 NCU_DRAM_BYTES_PER_COORD = {
     (15, 4, True): (1.040227e9 + 489.57e6) / 8388608,
+    (15, 2, True): (788.577e6 + 484.61e6) / 8388608,
 }
 
 
