@@ -473,6 +473,73 @@ cudaError_t launch_signum_push(const void* g, float* v, float beta, float omb, i
     return cudaGetLastError();
 }
 
+// Single-worker signSGD (Theorem 1's update, x <- x - eta sign(g); M = 1, no momentum): no vote to
+// take, so the step is sign packing and the parameter update in one lean pass: per quad one
+// gradient load, one parameter load, the sign nibble, the update, one store, and the packed word
+// by an OR tree. `flip` complements the signs (the lone worker is an inverting adversary).
+template <typename GT, int U>
+__global__ void __launch_bounds__(256)
+single_worker_kernel(const void* __restrict__ g, float* __restrict__ x, uint32_t* __restrict__ words,
+                     int64_t d, float lr, float wd, uint32_t flip) {
+    const int lane = threadIdx.x & 31;
+    const int k = lane & 7;
+    const int64_t n_quads = (d >> 5) << 3;
+    const int64_t tile = static_cast<int64_t>(blockDim.x) * U;
+    const bool has_wd = wd != 0.0f;
+    const uint32_t fn = flip ? 0xFu : 0u;
+    for (int64_t base = static_cast<int64_t>(blockIdx.x) * tile; base < n_quads;
+         base += static_cast<int64_t>(gridDim.x) * tile) {
+        float4 gq[U], xq[U];
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const int64_t q = base + static_cast<int64_t>(u) * blockDim.x + threadIdx.x;
+            const bool ok = q < n_quads;
+            gq[u] = ok ? GT::load4(g, q) : make_float4(-1.f, -1.f, -1.f, -1.f);
+            xq[u] = ok ? __ldcs(reinterpret_cast<const float4*>(x) + q) : make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const int64_t q = base + static_cast<int64_t>(u) * blockDim.x + threadIdx.x;
+            const bool ok = q < n_quads;
+            const uint32_t nib = ok ? (sign_nibble(gq[u]) ^ fn) : 0u;
+            if (ok) __stcs(reinterpret_cast<float4*>(x) + q, update_rn4(xq[u], nib, lr, wd, has_wd));
+            if (words != nullptr) {
+                uint32_t w = nib << (4 * k);
+                w |= __shfl_xor_sync(0xFFFFFFFFu, w, 1);
+                w |= __shfl_xor_sync(0xFFFFFFFFu, w, 2);
+                w |= __shfl_xor_sync(0xFFFFFFFFu, w, 4);
+                if (k == 0 && ok) words[q >> 3] = w;
+            }
+        }
+    }
+    if ((d & 31) != 0 && blockIdx.x == 0 && threadIdx.x < 32) {
+        const int64_t c = ((d >> 5) << 5) + lane;
+        const bool valid = c < d;
+        const float z = valid ? GT::load1(g, c) : -1.0f;
+        const uint32_t vmask = __ballot_sync(0xFFFFFFFFu, valid);
+        uint32_t w = __ballot_sync(0xFFFFFFFFu, valid && z >= 0.0f);
+        if (flip) w = ~w & vmask;
+        if (valid) x[c] = update_rn(x[c], (w >> lane) & 1u, lr, wd, has_wd);
+        if (lane == 0 && words != nullptr) words[d >> 5] = w;
+    }
+}
+
+template <typename GT>
+cudaError_t launch_single_worker(const StepDesc& s, cudaStream_t st) {
+    int threads = launch_options().threads > 0 ? launch_options().threads : 256;
+    if (threads > 256) threads = 256;
+    constexpr int U = 4;
+    auto kernel = single_worker_kernel<GT, U>;
+    const int64_t quads = (s.d >> 5) << 3;
+    const int64_t tile = static_cast<int64_t>(threads) * U;
+    int grid = 1;
+    cudaError_t err = pick_grid(kernel, threads, (quads + tile - 1) / tile, &grid);
+    if (err != cudaSuccess) return err;
+    kernel<<<grid, threads, 0, st>>>(s.g[0], s.x, s.words, s.d, s.lr, s.wd,
+                                     static_cast<uint32_t>(s.flip & 1ull));
+    return cudaGetLastError();
+}
+
 template <int M_CT, typename GT, bool MOM, bool APPLY, bool VEC, bool SEG = false>
 cudaError_t launch_step_inst(const StepDesc& s, cudaStream_t st) {
     using S = StepShape<M_CT, MOM>;
@@ -548,6 +615,7 @@ cudaError_t launch_step_dtype(const StepDesc& s, cudaStream_t st) {
 #undef SS_STEP_PICK_SEG
     }
     if (!s.vec) return SS_STEP_PICK(0, true, false);
+    if (s.M == 1 && !mom) return launch_single_worker<GT>(s, st);
     switch (s.M) {
         case 1: return SS_STEP_PICK(1, true, true);
         case 3: return SS_STEP_PICK(3, true, true);

@@ -429,3 +429,17 @@ def test_unfused_chain_replays_from_a_cuda_graph():
         assert torch.equal(x_g.view(torch.int32), x_e.view(torch.int32))
         for a, b in zip(mom_g, mom_e):
             assert torch.equal(a.view(torch.int32), b.view(torch.int32))
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16], ids=["f32", "bf16"])
+@pytest.mark.parametrize("flip,wd", [(0, 0.0), (1, 0.0), (0, 0.05), (1, 0.05)])
+@pytest.mark.parametrize("d,misalign", [(1, 0), (33, 0), (4097, 0), (4097, 1), (100_003, 0), (32 * 4096 + 8, 0)])
+def test_single_worker_signsgd_step(d, misalign, flip, wd, dtype):
+    """M = 1 without momentum (Theorem 1's update) has a kernel of its own."""
+    _fused_case(1, d, dtype, False, flip, wd, misalign, steps=2, seed=900 + d)
+    g = _rand(d, 950 + d, dtype)
+    xa = _rand(d, 951 + d, specials=False)
+    xb = xa.clone()
+    B.ss_fused_step([g], None, xa, 0.0, 1e-3, wd, flip, words_tensor(d, DEV))
+    B.ss_fused_step([g], None, xb, 0.0, 1e-3, wd, flip, None)       # without the packed output
+    assert torch.equal(xa.view(torch.int32), xb.view(torch.int32))
