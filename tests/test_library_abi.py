@@ -113,3 +113,22 @@ def test_missing_library_fails_loudly(monkeypatch, tmp_path):
     monkeypatch.setattr(B, "LIB_PATH", str(tmp_path / "libsignsgd.so"))
     with pytest.raises(RuntimeError, match="no CPU or PyTorch fallback"):
         B.ss_packed_words(5)
+
+
+def test_the_product_never_reaches_for_the_cpu_checker():
+    """The CPU oracle is test infrastructure: nothing under the package may import, load or name it,
+    and the binding must refuse to run without the CUDA library rather than fall back."""
+    pkg = os.path.join(ROOT, "paper_1810_05291_b200")
+    for dirpath, _, files in os.walk(pkg):
+        for fn in files:
+            if fn.endswith((".py", ".cu", ".cuh", ".h")):
+                text = open(os.path.join(dirpath, fn)).read()
+                assert "oracle" not in text.lower(), "%s mentions the oracle" % fn
+    missing = os.path.join(pkg, "no_such_dir", "libsignsgd.so")
+    saved_path, saved_lib = B.LIB_PATH, B._lib
+    try:
+        B.LIB_PATH, B._lib = missing, None
+        with pytest.raises(RuntimeError):
+            B.lib()
+    finally:
+        B.LIB_PATH, B._lib = saved_path, saved_lib
