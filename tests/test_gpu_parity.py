@@ -443,3 +443,39 @@ def test_single_worker_signsgd_step(d, misalign, flip, wd, dtype):
     B.ss_fused_step([g], None, xa, 0.0, 1e-3, wd, flip, words_tensor(d, DEV))
     B.ss_fused_step([g], None, xb, 0.0, 1e-3, wd, flip, None)       # without the packed output
     assert torch.equal(xa.view(torch.int32), xb.view(torch.int32))
+
+
+@pytest.mark.parametrize("threads,blocks_per_sm", [(128, 0), (64, 1), (256, 2), (192, 3)])
+def test_results_do_not_depend_on_the_launch_shape(threads, blocks_per_sm):
+    """Block size and the persistent-grid option change only how the tiles are walked."""
+    try:
+        B.ss_set_launch_option("threads", threads)
+        B.ss_set_launch_option("blocks_per_sm", blocks_per_sm)
+        d = 148 * 3 * 256 * 4 * 5 + 32 * 7 + 8       # several grid-stride rounds and a ragged word
+        _fused_case(15, d, torch.float32, True, 0b100, 0.0, 0, steps=1, seed=1234)
+        _fused_case(7, d, torch.bfloat16, False, 0, 0.01, 0, steps=1, seed=1235)
+        _fused_case(1, d, torch.float32, False, 0, 0.0, 0, steps=1, seed=1236)
+        _fused_case(5, 100_003, torch.float32, True, 0, 0.0, 1, steps=1, seed=1237)
+        g = _rand(d, 1238, torch.bfloat16)
+        out = words_tensor(d, DEV, fill=-1)
+        B.ss_sign_pack(g, out)
+        assert_words_equal(out, oracle.sign_pack(to_np(g)))
+        W = B.ss_packed_words(d)
+        gen = torch.Generator(device=DEV).manual_seed(1239)
+        packed = [torch.randint(-(1 << 31), 1 << 31, (W,), generator=gen, device=DEV,
+                                dtype=torch.int64).to(torch.int32) for _ in range(7)]
+        x = _rand(d, 1240, specials=False)
+        x_np = to_np(x)
+        vote = words_tensor(d, DEV, fill=-1)
+        B.ss_vote_apply(packed, x, 1e-3, 0.0, 0b1, vote)
+        want = oracle.majority_vote([to_np(p) for p in packed], d, 0b1)
+        oracle.apply_vote(x_np, want, 1e-3, 0.0)
+        assert_words_equal(vote, want)
+        assert count_bit_mismatch(x, x_np) == 0
+        tally = torch.zeros(d, dtype=torch.int8, device=DEV)
+        B.ss_vote_tally(packed, d, 0b1, tally)
+        assert np.array_equal(tally.cpu().numpy().astype(np.int32),
+                              oracle.majority_vote([to_np(p) for p in packed], d, 0b1, return_tally=True)[1])
+    finally:
+        B.ss_set_launch_option("threads", 0)
+        B.ss_set_launch_option("blocks_per_sm", 0)
