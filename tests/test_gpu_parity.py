@@ -479,3 +479,30 @@ def test_results_do_not_depend_on_the_launch_shape(threads, blocks_per_sm):
     finally:
         B.ss_set_launch_option("threads", 0)
         B.ss_set_launch_option("blocks_per_sm", 0)
+
+
+def test_two_streams_run_independent_steps_side_by_side():
+    """The library keeps no state between calls, so steps on different streams and buffers may
+    overlap on the GPU."""
+    M, d = 7, 32 * 60_000 + 8
+    sets = []
+    for k in range(2):
+        grads = [_rand(d, 9000 + 10 * k + m, specials=False) for m in range(M)]
+        x = _rand(d, 9100 + k, specials=False)
+        moms = [torch.zeros(d, device=DEV) for _ in range(M)]
+        sets.append((grads, moms, x, words_tensor(d, DEV), to_np(x), [np.zeros(d, dtype=np.float32) for _ in range(M)]))
+    streams = [torch.cuda.Stream(), torch.cuda.Stream()]
+    for s in streams:
+        s.wait_stream(torch.cuda.current_stream())
+    for step in range(4):
+        for k, s in enumerate(streams):
+            grads, moms, x, vote, _, _ = sets[k]
+            with torch.cuda.stream(s):
+                B.ss_fused_step(grads, moms, x, 0.9, 1e-3, 0.0, 0, vote)
+    torch.cuda.synchronize()
+    for grads, moms, x, vote, x_np, m_np in sets:
+        g_np = [to_np(g) for g in grads]
+        for step in range(4):
+            want = oracle.fused_step(g_np, m_np, x_np, 0.9, 1e-3)
+        assert_words_equal(vote, want)
+        assert count_bit_mismatch(x, x_np) == 0
