@@ -432,7 +432,9 @@ def main() -> None:
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="cfg3")
-    ap.add_argument("--d", type=int, default=None, help="override the coordinate count (tests, profiling)")
+    ap.add_argument("--d", "--coords", dest="d", type=int, default=None,
+                    help="override the coordinate count (tests, profiling); --coords is the spelling to use "
+                         "under torchrun, whose own parser finds --d ambiguous")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--profile", action="store_true",
