@@ -324,6 +324,8 @@ def table_mode(args) -> None:
         names = args.table.split(",")
         entries = ["pack", "signum_update", "vote", "apply", "vote_apply", "chain", "chain_va",
                    "chain_va_graph", "fused", "fused_segments"]
+    if args.entries:
+        entries = args.entries.split(",")
     rows = []
     for name in names:
         case = make_case(name, args.d)
@@ -442,6 +444,8 @@ def main() -> None:
     ap.add_argument("--table", default=None,
                     help="time every entry point: 'named' (cfg1-4), 'sweep' (the d x M sweep) or a "
                          "comma-separated list of workloads; one JSON line per row, then a table")
+    ap.add_argument("--entries", default=None,
+                    help="with --table: comma-separated entry points to time instead of the table's own list")
     ap.add_argument("--threads", type=int, default=0, help="launch-shape override: block size")
     ap.add_argument("--blocks-per-sm", type=int, default=0, help="launch-shape override")
     args = ap.parse_args()

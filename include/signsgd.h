@@ -29,7 +29,9 @@
  *              as host memory. Arrays of pointers (grads, momenta, packed) are HOST arrays of M
  *              device pointers; they are read during the call and may be freed after it returns.
  *              The library allocates no device memory and never frees or keeps a caller pointer.
- *              Buffers must not overlap each other; momentum and param are updated in place.
+ *              No buffer that a call writes (momenta, param, packed or vote words, staging) may
+ *              overlap any other buffer of the call; momentum and param are updated in place.
+ *              Read-only inputs may alias one another (two workers with the same gradient).
  * Alignment.   Word buffers: 4 bytes. Gradients: their element size. fp32 state: 4 bytes. When
  *              every gradient, momentum and parameter pointer of a call is 16-byte aligned
  *              (8-byte for bf16 gradients) the 128-bit vectorised kernels run; otherwise a
@@ -38,9 +40,11 @@
  * Streams.     cuda_stream is a cudaStream_t (NULL = the legacy default stream). Calls enqueue
  *              work on it and return without synchronising. The device that is current when
  *              the call is made is used.
- * Limits.      1 <= M <= SS_MAX_WORKERS. d >= 0; d == 0 is a no-op that returns SS_OK.
+ * Limits.      1 <= M <= SS_MAX_WORKERS. 0 <= d <= SS_MAX_COORDS; d == 0 is a no-op that returns
+ *              SS_OK, a d beyond the limit is SS_ERR_INVALID_ARG.
  * Errors.      Every function returns an int status: SS_OK (0) or a negative SS_ERR_* code;
- *              nothing is thrown across the boundary. On an argument error nothing is enqueued.
+ *              nothing is thrown across the boundary. Every argument of a call is checked before
+ *              its first copy or kernel is enqueued: on an argument error nothing is enqueued.
  *              SS_ERR_CUDA reports a failed launch or runtime call; ss_last_cuda_error() gives
  *              its cudaError_t value for the calling thread.
  */
@@ -54,6 +58,7 @@ extern "C" {
 #endif
 
 #define SS_MAX_WORKERS 64
+#define SS_MAX_COORDS ((int64_t)1 << 40) /* keeps every byte count formed from d inside 64 bits */
 
 typedef enum { SS_F32 = 0, SS_BF16 = 1 } ss_dtype;
 
@@ -119,7 +124,9 @@ int ss_signum_update(const void* grad, ss_dtype dt, float* momentum, float beta,
  * produces it. With one worker per GPU the destinations are the slot reserved for this worker
  * in every worker's receive buffer -- its own and its peers', mapped into this process with
  * peer access enabled -- so that the all-gather of packed words needs no separate collective.
- * Only plain stores go to a peer; nothing is read from one. The caller orders the exchange:
+ * Only plain stores go to a peer; nothing is read from one, whatever the alignment of grad and
+ * momentum (off the 16-byte grid a scalar-load kernel runs and stores to every destination
+ * itself). The caller orders the exchange:
  * every worker's call must have completed (stream synchronisation plus a barrier across the
  * workers) before any worker's ss_vote_apply reads its receive buffer, and the next step's push
  * must not start before those reads have finished.
@@ -252,10 +259,13 @@ int ss_fused_step_host(const void* const* host_grads, ss_dtype dt, void* const* 
  *
  * Limit: M * round_up(d * element size, 256) <= SS_STATIC_STAGING_BYTES. A larger request returns
  * SS_ERR_UNSUPPORTED and enqueues nothing; split the coordinates into ranges and call once per range.
- * The call itself performs no cudaMalloc, cudaFree or other allocating call.
  * First call on a device: it looks up the device address of the staging array (once per device,
- * with that device current) and keeps it. Make that first call during start-up, outside any
- * stream capture.
+ * with that device current) and keeps it. With lazy module loading, the CUDA default, that
+ * look-up is also what loads this part of the library onto the device, so it is then that the
+ * SS_STATIC_STAGING_BYTES are reserved; if the device has no room left for them the call returns
+ * SS_ERR_CUDA. Make that first call during start-up, before the device's memory is handed away
+ * and outside any stream capture. Every later call on that device performs no cudaMalloc,
+ * cudaFree or other allocating call and leaves the amount of free device memory unchanged.
  * Sharing: all calls on a device use the same staging array, and it keeps whatever the last call
  * left there. Every byte a call reads is first overwritten by that call's own copies, so nothing
  * needs clearing; but two calls whose work overlaps on the GPU (different streams, no dependency)
@@ -269,10 +279,13 @@ int ss_fused_step_host_static(const void* const* host_grads, ss_dtype dt, float*
                               uint32_t* host_vote_out, void* cuda_stream);
 
 /*
- * Launch-shape override for benchmarking sweeps (process-wide; not part of the method).
- *   key: "threads" (block size, multiple of 32 in [64, 1024], 0 = default) or
+ * Launch-shape override for benchmarking sweeps: not part of the method, and the one piece of
+ * process-wide state in the library (two integers, written and read atomically; a launch uses the
+ * values it finds when it is made, so change them only between calls whose shape matters).
+ *   key: "threads" (block size: a multiple of 32 in [64, 256], the bound the kernels are compiled
+ *        for; 0 = default, 256) or
  *        "blocks_per_sm" (0 = one block per tile, the default; n > 0 = a persistent grid of
-        n blocks per SM that strides over the tiles; at most 4096).
+ *        n blocks per SM that strides over the tiles; at most 4096).
  * Returns SS_ERR_INVALID_ARG for an unknown key or a value out of range.
  */
 int ss_set_launch_option(const char* key, int value);

@@ -118,11 +118,10 @@ __device__ __forceinline__ float4 update_seg4(const ss_segment* seg, int n, int6
 
 // ---- host side --------------------------------------------------------------------------
 
-struct LaunchOptions {
-    int threads = 0;        // 0: kernel default
-    int blocks_per_sm = 0;  // 0: one block per tile; > 0: persistent grid of this many blocks per SM
-};
-LaunchOptions& launch_options();
+// Launch-shape overrides (ss_set_launch_option): process-wide, read atomically at every launch.
+constexpr int kMaxBlockThreads = 256;  // every kernel is compiled with __launch_bounds__(256)
+int launch_threads();        // block size to use: the "threads" option, or 256 when it is 0
+int launch_blocks_per_sm();  // 0: one block per tile; > 0: persistent grid of this many blocks per SM
 int device_sm_count(cudaError_t* err);
 
 // Grid size for a grid-stride kernel. Default: one block per tile. On B200 the hardware block
@@ -133,7 +132,7 @@ template <typename Kernel>
 inline cudaError_t pick_grid(Kernel kernel, int threads, int64_t blocks_needed, int* grid_out) {
     (void)kernel;
     int64_t grid = blocks_needed;
-    const int per_sm = launch_options().blocks_per_sm;
+    const int per_sm = launch_blocks_per_sm();
     if (per_sm > 0) {
         cudaError_t err = cudaSuccess;
         const int sms = device_sm_count(&err);
@@ -163,12 +162,19 @@ struct StepDesc {
     int n_seg = 0;
 };
 
+// abi.cu: every argument check of a step, with no CUDA call (on SS_OK *out describes the launch;
+// out->d == 0 means nothing to do), and the launch of a checked step
+int validate_step(const void* const* grads, ss_dtype dt, float* const* momenta, int M, int64_t d,
+                  float beta, uint64_t flip_mask, float* param, float lr, float weight_decay,
+                  uint32_t* words, const ss_segment* seg, int n_seg, StepDesc* out);
+int launch_step(const StepDesc& s, ss_dtype dt, void* cuda_stream);
+
 cudaError_t launch_step_f32(const StepDesc& s, cudaStream_t st);
 cudaError_t launch_step_bf16(const StepDesc& s, cudaStream_t st);
 cudaError_t launch_signum_push_f32(const void* g, float* v, float beta, float omb, int64_t d,
-                                   uint32_t* const* dests, int n, cudaStream_t st);
+                                   uint32_t* const* dests, int n, bool vec, cudaStream_t st);
 cudaError_t launch_signum_push_bf16(const void* g, float* v, float beta, float omb, int64_t d,
-                                    uint32_t* const* dests, int n, cudaStream_t st);
+                                    uint32_t* const* dests, int n, bool vec, cudaStream_t st);
 cudaError_t launch_vote(const uint32_t* const* packed, int M, int64_t d, uint64_t flip,
                         uint32_t* vote, bool vec, cudaStream_t st);
 cudaError_t launch_vote_apply(const uint32_t* const* packed, int M, int64_t d, uint64_t flip,

@@ -6,7 +6,7 @@
 namespace ss {
 cudaError_t launch_step_f32(const StepDesc& s, cudaStream_t st) { return launch_step_dtype<F32>(s, st); }
 cudaError_t launch_signum_push_f32(const void* g, float* v, float beta, float omb, int64_t d,
-                                   uint32_t* const* dests, int n, cudaStream_t st) {
-    return launch_signum_push<F32>(g, v, beta, omb, d, dests, n, st);
+                                   uint32_t* const* dests, int n, bool vec, cudaStream_t st) {
+    return launch_signum_push<F32>(g, v, beta, omb, d, dests, n, vec, st);
 }
 }  // namespace ss

@@ -368,8 +368,7 @@ pack_ballot_kernel(const void* __restrict__ g, uint32_t* __restrict__ words, int
 
 template <typename GT>
 cudaError_t launch_pack(const StepDesc& s, cudaStream_t st) {
-    int threads = launch_options().threads > 0 ? launch_options().threads : 256;
-    if (threads > 256) threads = 256;
+    const int threads = launch_threads();
     int grid = 1;
     cudaError_t err;
     if (GT::kBytes == 2 && (reinterpret_cast<uintptr_t>(s.g[0]) & 15) == 0) {
@@ -401,9 +400,9 @@ cudaError_t launch_pack(const StepDesc& s, cudaStream_t st) {
 
 // ss_signum_update with the all-gather of the packed words folded into the producing kernel:
 // every word is stored to n destination buffers, which may be other GPUs' memory mapped into
-// this process (plain peer stores over NVLink; no multicast, nothing is read from a peer). The
-// words are 1/96 of the bytes this kernel moves, so the remote stores ride along with the
-// momentum pass instead of a separate collective reading the words back from HBM.
+// this process (plain peer stores over NVLink; nothing is read from a peer). The words are 1/96
+// of the bytes this kernel moves, so the remote stores ride along with the momentum pass instead
+// of a separate collective reading the words back from HBM.
 struct PushDests {
     uint32_t* p[SS_MAX_WORKERS];
     int n;
@@ -454,14 +453,56 @@ signum_push_kernel(const void* __restrict__ g, float* __restrict__ v, float beta
     }
 }
 
+// The same for pointers that are only element-aligned: ballot form (lane l owns coordinate
+// 32 j + l), PACK_WORDS words per warp, every word stored to all destinations by the lane that
+// holds it. Plain stores only, as above.
+template <typename GT>
+__global__ void __launch_bounds__(256)
+signum_push_ballot_kernel(const void* __restrict__ g, float* __restrict__ v, float beta, float omb,
+                          int64_t d, const __grid_constant__ PushDests dst) {
+    const int lane = threadIdx.x & 31;
+    const int64_t W = (d + 31) >> 5;
+    const int64_t warps = (static_cast<int64_t>(gridDim.x) * blockDim.x) >> 5;
+    for (int64_t j0 = ((static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x) >> 5) * PACK_WORDS;
+         j0 < W; j0 += warps * PACK_WORDS) {
+        float gs[PACK_WORDS], vs[PACK_WORDS];
+#pragma unroll
+        for (int k = 0; k < PACK_WORDS; ++k) {
+            const int64_t c = ((j0 + k) << 5) + lane;
+            gs[k] = c < d ? GT::load1(g, c) : -1.0f;
+            vs[k] = c < d ? __ldcs(v + c) : 0.0f;
+        }
+        uint32_t mine = 0u;
+#pragma unroll
+        for (int k = 0; k < PACK_WORDS; ++k) {
+            const int64_t c = ((j0 + k) << 5) + lane;
+            const float s = momentum_rn(omb, gs[k], beta, vs[k]);
+            if (c < d) __stcs(v + c, s);
+            const uint32_t w = __ballot_sync(0xFFFFFFFFu, c < d && s >= 0.0f);
+            if (lane == k) mine = w;
+        }
+        if (lane < PACK_WORDS && j0 + lane < W)
+            for (int p = 0; p < dst.n; ++p) dst.p[p][j0 + lane] = mine;
+    }
+}
+
 template <typename GT>
 cudaError_t launch_signum_push(const void* g, float* v, float beta, float omb, int64_t d,
-                               uint32_t* const* dests, int n, cudaStream_t st) {
+                               uint32_t* const* dests, int n, bool vec, cudaStream_t st) {
     PushDests dst;
     for (int p = 0; p < SS_MAX_WORKERS; ++p) dst.p[p] = p < n ? dests[p] : nullptr;
     dst.n = n;
-    int threads = launch_options().threads > 0 ? launch_options().threads : 256;
-    if (threads > 256) threads = 256;
+    const int threads = launch_threads();
+    if (!vec) {
+        const int64_t W = (d + 31) >> 5;
+        const int64_t per_block = static_cast<int64_t>(threads / 32) * PACK_WORDS;
+        auto kernel = signum_push_ballot_kernel<GT>;
+        int grid = 1;
+        cudaError_t err = pick_grid(kernel, threads, (W + per_block - 1) / per_block, &grid);
+        if (err != cudaSuccess) return err;
+        kernel<<<grid, threads, 0, st>>>(g, v, beta, omb, d, dst);
+        return cudaGetLastError();
+    }
     constexpr int U = 4;
     auto kernel = signum_push_kernel<GT, U>;
     const int64_t quads = (d >> 5) << 3;
@@ -526,8 +567,7 @@ single_worker_kernel(const void* __restrict__ g, float* __restrict__ x, uint32_t
 
 template <typename GT>
 cudaError_t launch_single_worker(const StepDesc& s, cudaStream_t st) {
-    int threads = launch_options().threads > 0 ? launch_options().threads : 256;
-    if (threads > 256) threads = 256;
+    const int threads = launch_threads();
     constexpr int U = 4;
     auto kernel = single_worker_kernel<GT, U>;
     const int64_t quads = (s.d >> 5) << 3;
@@ -560,8 +600,7 @@ cudaError_t launch_step_inst(const StepDesc& s, cudaStream_t st) {
     a.M = s.M;
     a.seg = s.seg;
     a.n_seg = s.n_seg;
-    int threads = launch_options().threads > 0 ? launch_options().threads : 256;
-    if (threads > 256) threads = 256;
+    const int threads = launch_threads();
     int grid = 1;
     cudaError_t err;
     if constexpr (VEC) {

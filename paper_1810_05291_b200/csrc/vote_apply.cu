@@ -144,8 +144,7 @@ cudaError_t launch_vote_inst(const uint32_t* const* packed, int M, int64_t d, ui
     a.d = d;
     a.flip = flip;
     a.M = M;
-    int threads = launch_options().threads > 0 ? launch_options().threads : 256;
-    if (threads > 256) threads = 256;
+    const int threads = launch_threads();
     const int64_t W = (d + 31) >> 5;
     int grid = 1;
     cudaError_t err;
@@ -307,8 +306,7 @@ cudaError_t launch_vote_apply_inst(const uint32_t* const* packed, int M, int64_t
     a.seg = seg;
     a.n_seg = n_seg;
     a.M = M;
-    int threads = launch_options().threads > 0 ? launch_options().threads : 256;
-    if (threads > 256) threads = 256;
+    const int threads = launch_threads();
     const int64_t tiles = (((d + 31) >> 5) + 31) >> 5;
     const int64_t per_block = threads / 32;
     int grid = 1;
@@ -441,8 +439,7 @@ cudaError_t launch_tally_inst(const uint32_t* const* packed, int M, int64_t d, u
     a.flip = flip;
     a.M = M;
     a.out_aligned4 = (reinterpret_cast<uintptr_t>(out) & 3) == 0;
-    int threads = launch_options().threads > 0 ? launch_options().threads : 256;
-    if (threads > 256) threads = 256;
+    const int threads = launch_threads();
     const int64_t tiles = (((d + 31) >> 5) + 31) >> 5;
     const int64_t per_block = threads / 32;
     int grid = 1;
@@ -531,8 +528,7 @@ cudaError_t launch_apply(float* x, const uint32_t* vote, int64_t d, float lr, fl
                          const ss_segment* seg, int n_seg, cudaStream_t st) {
     ApplyArgs a{x, vote, d, lr, wd, seg, n_seg};
     const bool segmented = seg != nullptr;
-    int threads = launch_options().threads > 0 ? launch_options().threads : 256;
-    if (threads > 256) threads = 256;
+    const int threads = launch_threads();
     int grid = 1;
     cudaError_t err;
     if (vec) {

@@ -91,8 +91,73 @@ def test_argument_errors_are_reported_before_any_cuda_call(L):
     assert L.ss_majority_vote(arr1, 1, 0, 0, None, None) == B.SS_OK
 
 
+def test_host_entry_points_check_every_argument_before_the_first_copy(L):
+    """ss_fused_step_host and its static-staging sibling: a bad momentum, parameter or vote buffer
+    must be reported before any copy is enqueued. With fake pointers and no GPU in reach, a call
+    that got as far as a copy would come back as SS_ERR_CUDA (or crash) instead."""
+    vp = ctypes.c_void_p
+    d, M = 64, 2
+    host = (vp * M)(0x10000, 0x20000)
+    stage = (vp * M)(0x30000, 0x40000)
+    mom_ok = (vp * M)(0x50000, 0x60000)
+    x, vote = vp(0x70000), vp(0x80000)
+
+    def host_call(staging=stage, momenta=mom_ok, param=x, words=vote, dd=d, flip=0):
+        return L.ss_fused_step_host(host, 0, staging, momenta, M, dd, 0.9, flip, param, 0.1, 0.0, words, None, None)
+
+    def static_call(momenta=mom_ok, param=x, words=vote, dd=d, flip=0):
+        return L.ss_fused_step_host_static(host, 0, momenta, M, dd, 0.9, flip, param, 0.1, 0.0, words, None, None)
+
+    for call in (host_call, static_call):
+        assert call(momenta=(vp * M)(0x50000, None)) == B.SS_ERR_INVALID_ARG          # NULL momentum
+        assert call(momenta=(vp * M)(0x50002, 0x60000)) == B.SS_ERR_MISALIGNED        # below 4 bytes
+        assert call(momenta=(vp * M)(0x50000, 0x50080)) == B.SS_ERR_INVALID_ARG       # momenta overlap
+        assert call(momenta=(vp * M)(0x50000, 0x70040)) == B.SS_ERR_INVALID_ARG       # momentum on param
+        assert call(words=vp(0x50004)) == B.SS_ERR_INVALID_ARG                        # vote on a momentum
+        assert call(words=vp(0x70010)) == B.SS_ERR_INVALID_ARG                        # vote on param
+        assert call(words=vp(0x80002)) == B.SS_ERR_MISALIGNED
+        assert call(param=vp(0x70001)) == B.SS_ERR_MISALIGNED
+        assert call(flip=4) == B.SS_ERR_INVALID_ARG
+        assert call(dd=(1 << 62) + 5) == B.SS_ERR_INVALID_ARG                         # d that would wrap d * 4
+        assert call(dd=(1 << 40) + 1) == B.SS_ERR_INVALID_ARG
+    assert host_call(staging=(vp * M)(0x30000, None)) == B.SS_ERR_INVALID_ARG
+    assert host_call(staging=(vp * M)(0x30000, 0x30040)) == B.SS_ERR_INVALID_ARG      # staging overlap
+    assert host_call(staging=(vp * M)(0x30000, 0x50000)) == B.SS_ERR_INVALID_ARG      # staging on a momentum
+    assert host_call(staging=(vp * M)(0x30000, 0x7FFF0)) == B.SS_ERR_INVALID_ARG      # staging on the vote
+    # the static variant's size limit is tested without forming a product that could wrap
+    assert static_call(dd=(B.SS_STATIC_STAGING_BYTES // 4) // M + 64) == B.SS_ERR_UNSUPPORTED
+    assert static_call(dd=1 << 40) == B.SS_ERR_UNSUPPORTED
+
+
+def test_sizes_that_would_wrap_a_byte_count_are_refused(L):
+    fake = ctypes.c_void_p(0x1000)
+    arr1 = (ctypes.c_void_p * 1)(0x1000)
+    for d in ((1 << 62) + 8, (1 << 63) - 1, (1 << 40) + 1):
+        assert L.ss_sign_pack(fake, 0, d, fake, None) == B.SS_ERR_INVALID_ARG
+        assert L.ss_fused_step(arr1, 0, None, 1, d, 0.0, 0, fake, 0.1, 0.0, None, None) == B.SS_ERR_INVALID_ARG
+        assert L.ss_majority_vote(arr1, 1, d, 0, fake, None) == B.SS_ERR_INVALID_ARG
+        assert L.ss_apply_vote(fake, fake, d, 0.1, 0.0, None) == B.SS_ERR_INVALID_ARG
+        assert L.ss_vote_apply(arr1, 1, d, 0, fake, 0.1, 0.0, None, None) == B.SS_ERR_INVALID_ARG
+        assert L.ss_signum_update_push(fake, 0, fake, 0.9, d, arr1, 1, None) == B.SS_ERR_INVALID_ARG
+        assert L.ss_vote_tally(arr1, 1, d, 0, fake, None) == B.SS_ERR_INVALID_ARG
+
+
+def test_step_arguments_may_not_alias_what_the_step_writes(L):
+    vp = ctypes.c_void_p
+    g = (vp * 2)(0x10000, 0x20000)
+    x = vp(0x70000)
+    # a momentum buffer on another worker's gradient
+    assert L.ss_fused_step(g, 0, (vp * 2)(0x50000, 0x10040), 2, 64, 0.9, 0, x, 0.1, 0.0, None, None) == B.SS_ERR_INVALID_ARG
+    # the packed output of ss_signum_update on its momentum
+    assert L.ss_signum_update(vp(0x10000), 0, vp(0x50000), 0.9, 64, vp(0x50010), None) == B.SS_ERR_INVALID_ARG
+
+
 def test_launch_option_validation(L):
     assert L.ss_set_launch_option(b"threads", 100) == B.SS_ERR_INVALID_ARG
+    assert L.ss_set_launch_option(b"threads", 512) == B.SS_ERR_INVALID_ARG      # kernels are built for <= 256
+    assert L.ss_set_launch_option(b"threads", 1024) == B.SS_ERR_INVALID_ARG
+    assert L.ss_set_launch_option(b"threads", 256) == B.SS_OK
+    assert L.ss_set_launch_option(b"blocks_per_sm", 4097) == B.SS_ERR_INVALID_ARG
     assert L.ss_set_launch_option(b"nope", 1) == B.SS_ERR_INVALID_ARG
     assert L.ss_set_launch_option(None, 1) == B.SS_ERR_INVALID_ARG
     assert L.ss_set_launch_option(b"threads", 128) == B.SS_OK

@@ -10,12 +10,14 @@ The file name sorts last so that a run that stops at the first failure has alrea
 """
 import ctypes
 
+import numpy as np
 import pytest
 import torch
 
+import oracle
 from paper_1810_05291_b200 import binding as B
 from paper_1810_05291_b200 import inputs
-from tests.util import assert_f32_close, to_np
+from tests.util import assert_f32_close, assert_words_equal, count_bit_mismatch, to_np
 
 DEV = "cuda:0"
 
@@ -57,6 +59,63 @@ def test_static_staging_matches_caller_staging_on_two_calls_in_a_row():
     _run_pair(M=15, d=32 * 9000 + 8, dtype=torch.float32, momentum=True, flip=0, step=0)
     _run_pair(M=7, d=100_003, dtype=torch.bfloat16, momentum=True, flip=0x10, step=1)
     _run_pair(M=3, d=4097, dtype=torch.float32, momentum=False, flip=0, step=2)
+
+
+def _run_against_the_checker(M, d, dtype, flip, step, x, moms, x_np, moms_np):
+    """One static-staging step on the device and the same step in the CPU checker, compared
+    element by element: packed vote (on the device and as copied to the host), parameters, momenta."""
+    case = inputs.cfg3(d)
+    case.M, case.dtype = M, dtype
+    grads = inputs.gradients(case, DEV, step)
+    host = [g.cpu().pin_memory() for g in grads]
+    W = B.ss_packed_words(d)
+    vote = torch.full((W,), -1, dtype=torch.int32, device=DEV)
+    hv = torch.full((W,), -1, dtype=torch.int32).pin_memory()
+    B.ss_fused_step_host_static(host, moms, x, 0.9, 1e-4, 0.0, flip, vote, hv)
+    torch.cuda.synchronize()
+    want = oracle.fused_step([to_np(g) for g in grads], moms_np, x_np, 0.9, 1e-4, 0.0, flip)
+    assert_words_equal(vote, want, "packed vote")
+    assert np.array_equal(hv.numpy().view(np.uint32), want), "vote copied to the host"
+    assert_f32_close(x, x_np, "parameters")
+    assert count_bit_mismatch(x, x_np) == 0
+    for v, v_np in zip(moms, moms_np):
+        assert_f32_close(v, v_np, "momentum")
+        assert count_bit_mismatch(v, v_np) == 0
+
+
+@pytest.mark.gpu
+def test_static_staging_matches_the_cpu_checker_and_takes_no_device_memory():
+    """Two calls in a row with different shapes against the CPU checker directly, and the property
+    the entry point exists for: once the first call on the device has been made, further calls
+    leave the amount of free device memory exactly where it was."""
+    shapes = [(15, 32 * 9000 + 8, torch.float32, 0), (5, 77_777, torch.bfloat16, 0b00100)]
+    state = []
+    for M, d, dtype, flip in shapes:
+        x = torch.randn(d, device=DEV, generator=torch.Generator(device=DEV).manual_seed(d))
+        moms = [torch.zeros(d, device=DEV) for _ in range(M)]
+        state.append((x, moms, to_np(x), [np.zeros(d, dtype=np.float32) for _ in range(M)]))
+    (M, d, dtype, flip), (x, moms, x_np, moms_np) = shapes[0], state[0]
+    _run_against_the_checker(M, d, dtype, flip, 0, x, moms, x_np, moms_np)   # also the set-up call
+    host_sets = []
+    for (M, d, dtype, flip) in shapes:               # host buffers made before the measurement
+        case = inputs.cfg3(d)
+        case.M, case.dtype = M, dtype
+        host_sets.append([g.cpu().pin_memory() for g in inputs.gradients(case, DEV, 7)])
+    votes = [torch.zeros(B.ss_packed_words(d), dtype=torch.int32, device=DEV) for (_, d, _, _) in shapes]
+    torch.cuda.synchronize()
+    free_before, _ = torch.cuda.mem_get_info()
+    for _ in range(3):
+        for (M, d, dtype, flip), (x, moms, _, _), host, vote in zip(shapes, state, host_sets, votes):
+            B.ss_fused_step_host_static(host, moms, x, 0.9, 1e-4, 0.0, flip, vote, None)
+    torch.cuda.synchronize()
+    free_after, _ = torch.cuda.mem_get_info()
+    assert free_after == free_before, "a call changed the free device memory by %d bytes" % (free_before - free_after)
+    # those calls moved the state; bring the checker's copy along, then compare once more per shape
+    for (M, d, dtype, flip), (x, moms, x_np, moms_np), host in zip(shapes, state, host_sets):
+        for _ in range(3):
+            oracle.fused_step([to_np(h) for h in host], moms_np, x_np, 0.9, 1e-4, 0.0, flip)
+    for step, ((M, d, dtype, flip), (x, moms, x_np, moms_np)) in enumerate(zip(shapes, state)):
+        _run_against_the_checker(M, d, dtype, flip, 20 + step, x, moms, x_np, moms_np)
 
 
 @pytest.mark.gpu

@@ -32,9 +32,9 @@ def assert_words_equal(got: torch.Tensor, want: np.ndarray, what: str = "words")
                              % (what, bad.size, want.size, bad[0], g[bad[0]], want[bad[0]]))
 
 
-def assert_f32_close(got: torch.Tensor, want: np.ndarray, what: str = "fp32 state"):
+def assert_f32_close(got, want: np.ndarray, what: str = "fp32 state"):
     """|delta| <= 1e-6 relative per element; NaNs must sit at the same places."""
-    g = to_np(got)
+    g = got if isinstance(got, np.ndarray) else to_np(got)
     assert g.shape == want.shape
     nan_g, nan_w = np.isnan(g), np.isnan(want)
     assert np.array_equal(nan_g, nan_w), "%s: NaN pattern differs" % what
@@ -54,9 +54,18 @@ def count_bit_mismatch(got: torch.Tensor, want: np.ndarray) -> int:
     """Elements whose fp32 bit patterns differ. A NaN on both sides counts as equal: the NaN
     payload is the one thing IEEE 754 leaves to the implementation (x86 keeps the operand's
     payload, the GPU returns the canonical NaN)."""
-    g = to_np(got)
+    g = got if isinstance(got, np.ndarray) else to_np(got)
     both_nan = np.isnan(g) & np.isnan(want)
     return int(np.count_nonzero((g.view(np.uint32) != want.view(np.uint32)) & ~both_nan))
+
+
+def assert_f32_state(got: torch.Tensor, want: np.ndarray, what: str = "fp32 state"):
+    """Both bars on one device-to-host copy: within 1e-6 relative per element, and (because both
+    sides run the same rounded operation sequence) bit-identical apart from NaN payloads."""
+    g = to_np(got)
+    assert_f32_close(g, want, what)
+    n = count_bit_mismatch(g, want)
+    assert n == 0, "%s: %d elements differ in their bit patterns" % (what, n)
 
 
 class GuardedWords:
