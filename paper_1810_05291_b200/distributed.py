@@ -50,7 +50,9 @@ class PackedExchange:
         self.d, self.world, self.rank, self.mode, self.group = int(d), world, rank, mode, group
         self.coll = collectives if collectives is not None else dist
         self.W = packed_words(d)
-        self.slice_words = -(-max(self.W, 1) // world)      # words per server slice
+        # words per server slice, rounded up to 4 so that every worker's row of the gathered
+        # buffer and every slice starts on a 16-byte boundary (the kernels' wide loads need it)
+        self.slice_words = 4 * -(-max(self.W, 1) // (4 * world))
         self.W_pad = self.slice_words * world               # local buffer, padded with zero words
         kw = dict(dtype=torch.int32, device=device)
         self.local = torch.zeros(self.W_pad, **kw)          # this worker's packed sign(v)

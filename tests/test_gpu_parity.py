@@ -216,6 +216,57 @@ def test_vote_apply(d, misalign, M):
         check_guard(full, lo, d)
 
 
+@pytest.mark.parametrize("M", [2, 6, 9, 14, 17, 27, 30, 33, 62])
+def test_vote_and_vote_apply_for_worker_counts_between_the_compiled_ones(M):
+    """Worker counts that have no kernel of their own run the next larger compiled capacity with
+    the absent workers switched off: vote, tally sign and parameters against the oracle."""
+    d = 64 * 32 * 5 + 32 * 3 + 5                       # full 64-word tiles, then a ragged end
+    W = B.ss_packed_words(d)
+    gen = torch.Generator(device=DEV).manual_seed(1000 + M)
+    packed = [torch.randint(-(1 << 31), 1 << 31, (W,), generator=gen, device=DEV,
+                            dtype=torch.int64).to(torch.int32) for _ in range(M)]
+    packed_np = [to_np(p) for p in packed]
+    flip = (0x5A5A5A5A5A5A5A5A >> 3) & ((1 << M) - 1)
+    want = oracle.majority_vote(packed_np, d, flip)
+    out = GuardedWords(d, DEV)
+    B.ss_majority_vote(packed, d, flip, out.view)
+    assert_words_equal(out.view, want, "ss_majority_vote")
+    out.check()
+    full, x, lo = guarded_f32(_rand(d, 900 + M, specials=False), 0)
+    x_np = to_np(x)
+    oracle.apply_vote(x_np, want, 1e-3, 0.01)
+    out2 = GuardedWords(d, DEV)
+    B.ss_vote_apply(packed, x, 1e-3, 0.01, flip, out2.view)
+    assert_words_equal(out2.view, want, "ss_vote_apply")
+    out2.check()
+    assert count_bit_mismatch(x, x_np) == 0
+    check_guard(full, lo, d)
+
+
+@pytest.mark.parametrize("M", [3, 15, 20, 64])
+@pytest.mark.parametrize("packed_off,vote_off", [(2, 0), (0, 2), (1, 0), (0, 1), (2, 2), (3, 1)])
+def test_vote_apply_with_packed_words_off_the_16_byte_grid(M, packed_off, vote_off):
+    """The parameters 16-byte aligned, the packed inputs or the vote output shifted by whole
+    words: 8-byte shifts keep the 64-bit loads, odd shifts take the word-at-a-time kernel."""
+    d = 64 * 32 * 7 + 32 * 40 + 9
+    W = B.ss_packed_words(d)
+    gen = torch.Generator(device=DEV).manual_seed(2000 + M + packed_off)
+    packed = [torch.randint(-(1 << 31), 1 << 31, (W + packed_off,), generator=gen, device=DEV,
+                            dtype=torch.int64).to(torch.int32)[packed_off:] for _ in range(M)]
+    packed_np = [to_np(p) for p in packed]
+    flip = 0b101 & ((1 << M) - 1)
+    want = oracle.majority_vote(packed_np, d, flip)
+    full, x, lo = guarded_f32(_rand(d, 950 + M, specials=False), 0)
+    x_np = to_np(x)
+    oracle.apply_vote(x_np, want, 1e-3, 0.0)
+    out = GuardedWords(d, DEV, misalign_words=vote_off)
+    B.ss_vote_apply(packed, x, 1e-3, 0.0, flip, out.view)
+    assert_words_equal(out.view, want)
+    out.check()
+    assert count_bit_mismatch(x, x_np) == 0
+    check_guard(full, lo, d)
+
+
 def test_vote_apply_equals_vote_then_apply_on_the_gpu():
     M, d = 15, 32 * 40_000 + 8
     gen = torch.Generator(device=DEV).manual_seed(77)
