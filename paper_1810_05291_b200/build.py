@@ -22,7 +22,7 @@ LIB = os.path.join(HERE, "libsignsgd.so")
 OBJ_DIR = os.path.join(ROOT, "_build", "signsgd")
 
 SOURCES = ["abi.cu", "step_f32.cu", "step_bf16.cu", "vote_apply.cu", "noalloc.cu"]
-HEADERS = ["bitslice.cuh", "common.cuh", "step_kernel.cuh", os.path.join("..", "..", "include", "signsgd.h")]
+HEADERS = ["bitslice.cuh", "common.cuh", "step_kernel.cuh", "step_oct_kernel.cuh", os.path.join("..", "..", "include", "signsgd.h")]
 
 # -fmad=false: no multiply-add contraction anywhere (the arithmetic also uses explicitly
 # rounded intrinsics); no -use_fast_math, denormals kept.

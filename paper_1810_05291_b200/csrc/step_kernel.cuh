@@ -580,13 +580,11 @@ cudaError_t launch_single_worker(const StepDesc& s, cudaStream_t st) {
     return cudaGetLastError();
 }
 
-template <int M_CT, typename GT, bool MOM, bool APPLY, bool VEC, bool SEG = false>
-cudaError_t launch_step_inst(const StepDesc& s, cudaStream_t st) {
-    using S = StepShape<M_CT, MOM>;
-    StepArgs<S::NP> a;
-    for (int m = 0; m < S::NP; ++m) {
+template <int NP>
+void fill_step_args(StepArgs<NP>& a, const StepDesc& s, bool mom) {
+    for (int m = 0; m < NP; ++m) {
         a.g[m] = m < s.M ? s.g[m] : nullptr;
-        a.v[m] = (MOM && m < s.M) ? s.v[m] : nullptr;
+        a.v[m] = (mom && m < s.M) ? s.v[m] : nullptr;
         a.fnib[m] = (m < s.M && ((s.flip >> m) & 1ull)) ? 0xFu : 0u;
     }
     a.x = s.x;
@@ -600,6 +598,13 @@ cudaError_t launch_step_inst(const StepDesc& s, cudaStream_t st) {
     a.M = s.M;
     a.seg = s.seg;
     a.n_seg = s.n_seg;
+}
+
+template <int M_CT, typename GT, bool MOM, bool APPLY, bool VEC, bool SEG = false>
+cudaError_t launch_step_inst(const StepDesc& s, cudaStream_t st) {
+    using S = StepShape<M_CT, MOM>;
+    StepArgs<S::NP> a;
+    fill_step_args(a, s, MOM);
     const int threads = launch_threads();
     int grid = 1;
     cudaError_t err;
@@ -624,10 +629,19 @@ cudaError_t launch_step_inst(const StepDesc& s, cudaStream_t st) {
 // dispatch on (M, momentum, apply, alignment) for one gradient dtype. The vector form is
 // specialised for the worker counts of the paper's experiments and of the sweep (all 2^k - 1,
 // plus 16 for the even-M probe); any other M, and every unaligned call, takes the runtime-M form.
+// bf16 gradients on 16-byte aligned pointers: the octet kernels (step_oct_kernel.cuh)
+template <bool SEG>
+cudaError_t launch_step_oct(const StepDesc& s, cudaStream_t st);
+
 template <typename GT>
 cudaError_t launch_step_dtype(const StepDesc& s, cudaStream_t st) {
     const bool mom = s.v != nullptr;
     const bool apply = s.x != nullptr;
+    if constexpr (GT::kBytes == 2) {
+        bool oct = s.vec && (apply || mom);  // plain sign packing has an octet kernel of its own
+        for (int m = 0; m < s.M; ++m) oct = oct && (reinterpret_cast<uintptr_t>(s.g[m]) & 15) == 0;
+        if (oct) return s.seg != nullptr ? launch_step_oct<true>(s, st) : launch_step_oct<false>(s, st);
+    }
 #define SS_STEP_PICK(MV, AP, VC)                                             \
     (mom ? launch_step_inst<MV, GT, true, AP, VC>(s, st)                     \
          : launch_step_inst<MV, GT, false, AP, VC>(s, st))

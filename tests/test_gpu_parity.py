@@ -97,7 +97,7 @@ def test_sign_pack(d, misalign, dtype):
 
 
 @pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16], ids=["f32", "bf16"])
-@pytest.mark.parametrize("misalign", [0, 1], ids=["aligned", "unaligned"])
+@pytest.mark.parametrize("misalign", [0, 1, 4], ids=["aligned", "unaligned", "off-by-4-elements"])
 @pytest.mark.parametrize("d", AWKWARD_D)
 def test_signum_update(d, misalign, dtype):
     g = _rand(d + misalign, 200 + d, dtype)[misalign:]
@@ -315,15 +315,16 @@ def _fused_case(M, d, dtype, momentum, flip, wd, misalign, steps=2, seed=0):
 
 @pytest.mark.parametrize("momentum", [False, True], ids=["signsgd", "signum"])
 @pytest.mark.parametrize("M", ALL_M)
-def test_fused_step_all_worker_counts(M, momentum):
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16], ids=["f32", "bf16"])
+def test_fused_step_all_worker_counts(M, momentum, dtype):
     flip = (0x5A5A5A5A5A5A5A5A if M > 2 else 0) & ((1 << M) - 1)
     if M % 2 == 1 and bin(flip).count("1") * 2 > M:
         flip = 0
-    _fused_case(M, 32 * 1024 * 3 + 8, torch.float32, momentum, flip, 0.0, 0, seed=M * 31)
+    _fused_case(M, 32 * 1024 * 3 + 8, dtype, momentum, flip, 0.0, 0, seed=M * 31)
 
 
 @pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16], ids=["f32", "bf16"])
-@pytest.mark.parametrize("misalign", [0, 1], ids=["aligned", "unaligned"])
+@pytest.mark.parametrize("misalign", [0, 1, 4], ids=["aligned", "unaligned", "off-by-4-elements"])
 @pytest.mark.parametrize("d", AWKWARD_D)
 @pytest.mark.parametrize("M,momentum", [(3, False), (15, True), (6, True)])
 def test_fused_step_awkward_shapes(d, misalign, dtype, M, momentum):

@@ -124,6 +124,31 @@ def test_fused_step_segments_matches_per_tensor_steps(M, momentum, d, n_seg, mis
 
 
 @pytest.mark.gpu
+@pytest.mark.parametrize("M,momentum", [(3, False), (15, True), (6, True)])
+@pytest.mark.parametrize("d,n_seg", [(4097, 5), (100_003, 161)])
+def test_fused_step_segments_with_bf16_gradients(M, momentum, d, n_seg):
+    """bf16 gradients on aligned pointers run kernels of their own (eight coordinates per thread);
+    the per-tensor learning rates must reach both quads of every octet."""
+    g32, v, x = _inputs(M, d, 20 * d + M, momentum)
+    gd = [torch.from_numpy(a).to(DEV).to(torch.bfloat16) for a in g32]
+    g = [t.cpu().view(torch.int16).numpy().view(np.uint16).copy() for t in gd]   # raw bf16 for the checker
+    begins, lrs, wds = _table(d, n_seg, d + n_seg + 1)
+    tab = B.segment_table(n_seg, DEV)
+    B.ss_segments_upload(begins, lrs, wds, d, tab)
+    vd = [_to_dev(a) for a in v] if momentum else None
+    xd = _to_dev(x)
+    vote = torch.full((B.ss_packed_words(d),), -1, dtype=torch.int32, device=DEV)
+    for step in range(2):
+        B.ss_fused_step_segments(gd, vd, xd, 0.9, tab, n_seg, 0b100, vote)
+        want = oracle.fused_step_segments(g, v, x, 0.9, begins, lrs, wds, 0b100)
+        assert np.array_equal(vote.cpu().numpy().view(np.uint32), want), "vote, step %d" % step
+        assert np.array_equal(xd.cpu().numpy().view(np.uint32), x.view(np.uint32)), "x, step %d" % step
+        if momentum:
+            for a, b in zip(vd, v):
+                assert np.array_equal(a.cpu().numpy().view(np.uint32), b.view(np.uint32))
+
+
+@pytest.mark.gpu
 @pytest.mark.parametrize("d,n_seg", [(1, 1), (127, 3), (100_003, 161)])
 @pytest.mark.parametrize("misalign", [0, 1], ids=["aligned", "unaligned"])
 def test_apply_vote_segments(d, n_seg, misalign):
