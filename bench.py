@@ -2,11 +2,18 @@
 """Benchmark of the fused Signum step (momentum -> sign -> majority vote -> update, one kernel).
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--workload cfg3] [--impl ours|reference]
+    python bench.py --mode worker-per-gpu --layout allgather|sharded|push [--gpus N]
+    python bench.py --table named|sweep|<workloads> [--entries ...]
 
 A step is one call of ss_fused_step over one batch of synthetic gradients: M = 15 workers,
-d = 25,557,032 (ResNet-50-sized) fp32, per-worker momentum, beta = 0.9, lr = 1e-4. Under
-torchrun every rank runs the same workload on its own GPU (the path shards by coordinate and
-needs no collective), timing is the maximum over ranks, and rank 0 prints one JSON line.
+d = 25,557,032 (ResNet-50-sized) fp32, per-worker momentum, beta = 0.9, lr = 1e-4. With more than
+one rank every rank runs the same workload on its own GPU (the path shards by coordinate and needs
+no collective), timing is the maximum over ranks, and rank 0 prints one JSON line. The ranks come
+from a launcher (torch.distributed.run sets RANK / LOCAL_RANK / WORLD_SIZE) or, when --gpus N is
+given to a plain process, from this script starting them itself.
+
+--mode worker-per-gpu measures the other multi-GPU form, Algorithm 1 with one worker per GPU and
+the packed signs exchanged between them, in three layouts of that exchange.
 """
 
 from __future__ import annotations
@@ -31,12 +38,30 @@ NOMINAL_HBM_GBS = 8000.0
 
 # DRAM bytes per coordinate (dram__bytes_read.sum + dram__bytes_write.sum) of the fused kernels,
 # from ncu captures at d = 8,388,608 (larger than L2; traffic is proportional to d because every
-# coordinate is touched exactly once). Keyed by (M, gradient bytes, momentum). An entry is
-# removed when its kernel changes until the counters are taken again.
+# coordinate is touched exactly once). Keyed by (M, gradient bytes, momentum). Each entry carries
+# the hash of the kernel sources at the time of the capture (kernel_source_hash below); when the
+# sources have changed since, the entry no longer describes the kernel that runs and
+# roofline.traffic is reported as null until the counters are taken again.
 NCU_DRAM_BYTES_PER_COORD = {
-    (15, 4, True): (1.040227e9 + 489.57e6) / 8388608,
-    (15, 2, True): (788.577e6 + 484.61e6) / 8388608,
+    (15, 4, True): {"bytes_per_coord": (1.040266e9 + 488.44e6) / 8388608, "capture_d": 8388608,
+                    "sources": "f32", "source_hash": "e4f57e4b37bb6d15"},
+    (15, 2, True): {"bytes_per_coord": (788.708e6 + 483.37e6) / 8388608, "capture_d": 8388608,
+                    "sources": "bf16", "source_hash": "0268b7e0c7ff236e"},
 }
+KERNEL_SOURCES = {
+    "f32": ("step_kernel.cuh", "bitslice.cuh", "common.cuh"),
+    "bf16": ("step_oct_kernel.cuh", "step_kernel.cuh", "bitslice.cuh", "common.cuh"),
+}
+
+
+def kernel_source_hash(which: str) -> str:
+    """sha256 (first 16 hex digits) over the sources that define the fused kernel of a gradient dtype."""
+    import hashlib
+    h = hashlib.sha256()
+    for name in KERNEL_SOURCES[which]:
+        with open(os.path.join(ROOT, "paper_1810_05291_b200", "csrc", name), "rb") as f:
+            h.update(f.read())
+    return h.hexdigest()[:16]
 
 
 def make_case(name: str, d_override=None):
@@ -73,12 +98,20 @@ def algorithmic_bytes(case) -> int:
 
 
 def ncu_traffic(case):
-    """DRAM bytes of one launch of the fused kernel on this workload, scaled from the ncu capture
-    of a smaller case of the same kernel; None when no capture of that kernel is on record."""
+    """(bytes, note): DRAM bytes of one launch of the fused kernel on this workload, scaled by d
+    from the recorded ncu capture of a smaller case of the same kernel; bytes is None when no
+    capture is on record or the kernel sources have changed since it was taken."""
     import torch
     key = (case.M, 4 if case.dtype == torch.float32 else 2, case.beta is not None)
-    per = NCU_DRAM_BYTES_PER_COORD.get(key)
-    return None if per is None else per * case.d
+    rec = NCU_DRAM_BYTES_PER_COORD.get(key)
+    if rec is None:
+        return None, "no ncu capture on record for this kernel"
+    now = kernel_source_hash(rec["sources"])
+    if now != rec["source_hash"]:
+        return None, ("kernel sources changed since the ncu capture (hash %s, capture %s): counters must be "
+                      "taken again" % (now, rec["source_hash"]))
+    return rec["bytes_per_coord"] * case.d, ("scaled by d from the recorded ncu capture at d=%d (sources %s)"
+                                             % (rec["capture_d"], now))
 
 
 def measured_peak():
@@ -96,8 +129,8 @@ class ClockSampler:
               "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
               "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
 
-    def __init__(self, index: int):
-        self.index = index
+    def __init__(self, index):
+        self.index = index          # what nvidia-smi -i accepts: an index or a GPU / MIG UUID
         self.proc = None
         self.lines = []
 
@@ -105,7 +138,7 @@ class ClockSampler:
         try:
             self.proc = subprocess.Popen(
                 ["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.FIELDS,
-                 "--format=csv,noheader,nounits", "-lms", "100"],
+                 "--format=csv,noheader,nounits", "-lms", "50"],
                 stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
             self.thread = threading.Thread(target=self._read, daemon=True)
             self.thread.start()
@@ -125,7 +158,7 @@ class ClockSampler:
             self.proc.wait(timeout=5)
         except Exception:
             self.proc.kill()
-        rows = [l for (t, l) in self.lines if t0 <= t <= t1 + 0.2] or [l for (_, l) in self.lines]
+        rows = [l for (t, l) in self.lines if t0 <= t <= t1] or [l for (_, l) in self.lines]
         sm, smax, power, reasons = [], [], [], set()
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
         for r in rows:
@@ -427,46 +460,98 @@ def table_mode(args) -> None:
             r["frac_of_measured_copy"]))
 
 
-def main() -> None:
-    ap = argparse.ArgumentParser()
-    ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=50)
-    ap.add_argument("--warmup", type=int, default=5)
-    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="cfg3")
-    ap.add_argument("--d", "--coords", dest="d", type=int, default=None,
-                    help="override the coordinate count (tests, profiling); --coords is the spelling to use "
-                         "under torchrun, whose own parser finds --d ambiguous")
-    ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--no-e2e", action="store_true")
-    ap.add_argument("--profile", action="store_true",
-                    help="for runs under a profiler: no clock sampling, no end-to-end and CPU legs")
-    ap.add_argument("--table", default=None,
-                    help="time every entry point: 'named' (cfg1-4), 'sweep' (the d x M sweep) or a "
-                         "comma-separated list of workloads; one JSON line per row, then a table")
-    ap.add_argument("--entries", default=None,
-                    help="with --table: comma-separated entry points to time instead of the table's own list")
-    ap.add_argument("--threads", type=int, default=0, help="launch-shape override: block size")
-    ap.add_argument("--blocks-per-sm", type=int, default=0, help="launch-shape override")
-    args = ap.parse_args()
-    if args.warmup < 3:
-        args.warmup = 3
-    if args.profile:
-        args.no_e2e = args.no_cpu_baseline = True
+def smi_device_id(local_rank: int) -> str:
+    """The id nvidia-smi knows this rank's GPU by: the rank's entry of CUDA_VISIBLE_DEVICES (an
+    index or a GPU-/MIG- UUID, passed on as text) or, without that variable, the local rank."""
+    vis = [v.strip() for v in os.environ.get("CUDA_VISIBLE_DEVICES", "").split(",") if v.strip()]
+    if local_rank < len(vis):
+        return vis[local_rank]
+    return str(local_rank)
 
-    if args.impl == "reference":
-        reference_arm(args)
-        return
-    if args.table:
-        table_mode(args)
-        return
 
+def free_port() -> int:
+    import socket
+    with socket.socket() as sock:
+        sock.bind(("127.0.0.1", 0))
+        return sock.getsockname()[1]
+
+
+def launch_command(n_ranks: int, argv, port: int):
+    """The command that runs this script as n_ranks processes on one node, one GPU each."""
+    return [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", "--nproc-per-node", str(n_ranks),
+            "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__)] + list(argv)
+
+
+def spawn_ranks(n_ranks: int, argv, run=subprocess.call) -> int:
+    """`bench.py --gpus N` started as a plain process: start the N ranks (the script itself under
+    torch.distributed.run, which sets RANK / LOCAL_RANK / WORLD_SIZE) and pass on their exit code.
+    --d is respelt --coords, the form torchrun's own parser leaves alone."""
+    argv = ["--coords" if a == "--d" else a for a in argv]
+    return run(launch_command(n_ranks, argv, free_port()))
+
+
+def launch_check_mode(args) -> None:
+    """--mode launch-check: every rank joins a gloo group on the CPU, the ranks are counted with an
+    all-reduce and rank 0 prints one line. Exercises the launcher without a GPU."""
     import torch
     import torch.distributed as dist
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    seen = world
+    if world > 1:
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        dist.init_process_group("gloo")
+        t = torch.ones(1, dtype=torch.int64)
+        dist.all_reduce(t)
+        seen = int(t.item())
+        dist.destroy_process_group()
+    if rank == 0:
+        print(json.dumps({"mode": "launch-check", "n_gpus": world, "ranks_seen": seen,
+                          "gpus_requested": args.gpus}), flush=True)
 
-    from paper_1810_05291_b200 import binding as B
-    from paper_1810_05291_b200 import inputs, sharding
 
+def timed_launches(step, steps: int, stream, barrier, per_launch: bool = False):
+    """EXACTLY `steps` calls of step() between a barrier + synchronize on both sides, timed by one
+    pair of CUDA events on the launching stream. With per_launch an event is also recorded after
+    every call, which gives the duration of every single launch from the same region.
+    Returns (total_ms, [per-launch ms] or None, host time at start, host time at end)."""
+    import torch
+    n_ev = steps + 1 if per_launch else 2
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(n_ev)]
+    barrier()
+    t0 = time.time()
+    ev[0].record(stream)
+    for i in range(steps):
+        step()
+        if per_launch:
+            ev[i + 1].record(stream)
+    if not per_launch:
+        ev[1].record(stream)
+    barrier()
+    t1 = time.time()
+    each = [ev[i].elapsed_time(ev[i + 1]) for i in range(steps)] if per_launch else None
+    return ev[0].elapsed_time(ev[-1]), each, t0, t1
+
+
+def keep_busy(step, seconds: float) -> None:
+    """Runs step() back to back for about `seconds`, so that the clock samples taken around the
+    timed region (itself too short for nvidia-smi to see) are samples of the GPU under this very load."""
+    import torch
+    t = time.time()
+    while time.time() - t < seconds:
+        for _ in range(50):
+            step()
+        torch.cuda.synchronize()
+
+
+def spread(ms) -> dict:
+    return {"ms_median": statistics.median(ms), "ms_min": min(ms), "ms_max": max(ms)}
+
+
+def init_ranks():
+    """(world, rank, local_rank, device) from the launcher's environment; NCCL group when world > 1."""
+    import torch
+    import torch.distributed as dist
     world = int(os.environ.get("WORLD_SIZE", "1"))
     rank = int(os.environ.get("RANK", "0"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
@@ -477,7 +562,18 @@ def main() -> None:
     if world > 1:
         os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
         dist.init_process_group("nccl", device_id=dev)
+    return world, rank, local_rank, dev
 
+
+def fused_mode(args) -> None:
+    """The default mode: one ss_fused_step per step on every rank's own coordinate shard."""
+    import torch
+    import torch.distributed as dist
+
+    from paper_1810_05291_b200 import binding as B
+    from paper_1810_05291_b200 import inputs, sharding
+
+    world, rank, local_rank, dev = init_ranks()
     B.lib()  # fail here, loudly, if the CUDA library is missing
     if args.threads:
         B.ss_set_launch_option("threads", args.threads)
@@ -504,33 +600,22 @@ def main() -> None:
     for _ in range(args.warmup):
         step()
     barrier()
-    sampler = ClockSampler(local_rank if "CUDA_VISIBLE_DEVICES" not in os.environ
-                           else int(os.environ["CUDA_VISIBLE_DEVICES"].split(",")[local_rank]))
+    sampler = ClockSampler(smi_device_id(local_rank))
+    busy = 0.0 if args.profile else 0.6
     if not args.profile:
         sampler.start()
-        time.sleep(0.3)
-        # a short spell of the same kernel so that clock samples are taken under load
-        for _ in range(args.warmup):
-            step()
-        barrier()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    t0 = time.time()
-    e0.record(stream)
-    for _ in range(args.steps):
-        step()
-    e1.record(stream)
-    barrier()
-    t1 = time.time()
-    ms_total = e0.elapsed_time(e1)
-    # keep the GPU busy a little longer if the timed region was too short for nvidia-smi to see
-    if t1 - t0 < 0.5 and not args.profile:
-        t_extra = time.time()
-        while time.time() - t_extra < 0.6:
-            for _ in range(20):
-                step()
-            torch.cuda.synchronize()
-        t1 = time.time()
-    clocks = sampler.stop(t0, t1) if not args.profile else {"sm_mhz": None, "reasons": ["not sampled (--profile)"]}
+        keep_busy(step, busy)          # the same kernel, back to back, before ...
+    ms_total, _, t0, t1 = timed_launches(step, args.steps, stream, barrier)
+    # the same K launches once more, straight after, now with an event after every launch: the
+    # spread of single launches, and a second total to hold against the first
+    ms_again, per_launch, _, t1 = timed_launches(step, args.steps, stream, barrier, per_launch=True)
+    if not args.profile:
+        keep_busy(step, busy)          # ... and after the timed launches
+    clocks = (sampler.stop(t0 - 0.8 * busy, t1 + 0.8 * busy) if not args.profile
+              else {"sm_mhz": None, "reasons": ["not sampled (--profile)"]})
+    if not args.profile:
+        clocks["window"] = ("samples every 50 ms while the same kernel runs back to back from %.1f s before "
+                            "to %.1f s after the timed launches" % (busy, busy))
 
     ms_total = sharding.max_over_ranks(ms_total, dev)
     ms_step = ms_total / args.steps
@@ -549,25 +634,22 @@ def main() -> None:
 
         for _ in range(2):
             step_host()
-        barrier()
-        h0, h1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        h0.record(stream)
-        for _ in range(n_e2e):
-            step_host()
-        h1.record(stream)
-        barrier()
-        ms_e2e = h0.elapsed_time(h1)
+        ms_e2e, per_e2e, _, _ = timed_launches(step_host, n_e2e, stream, barrier, per_launch=True)
         ms_e2e = sharding.max_over_ranks(ms_e2e, dev)
         e2e = {"value": world * case.d / (ms_e2e / n_e2e * 1e-3), "unit": UNIT,
                "h2d_bytes_per_step": sum(h.numel() * h.element_size() for h in host),
                "d2h_bytes_per_step": hv.numel() * 4, "steps": n_e2e,
-               "ms_per_step": ms_e2e / n_e2e, "entry_point": "ss_fused_step_host"}
+               "ms_per_step": ms_e2e / n_e2e, "entry_point": "ss_fused_step_host",
+               "result": "packed vote; x and v stay on the device"}
+        e2e.update(spread(per_e2e))
         del host
 
     if rank == 0:
         abytes = algorithmic_bytes(case)
         peak, peak_src = measured_peak()
         achieved = abytes / (ms_step * 1e-3) / 1e9
+        traffic, traffic_note = ncu_traffic(case)
+        sm_mhz = clocks.get("sm_mhz")
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True,
@@ -577,15 +659,25 @@ def main() -> None:
             "hbm_gbs": achieved, "pct_of_nominal_8tbs": 100.0 * achieved / NOMINAL_HBM_GBS,
             "gradient_elements_per_s": value * case.M,
             "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
-                         "frac": achieved / peak, "traffic": ncu_traffic(case), "peak_source": peak_src,
-                         "kernel": "step_vec_kernel<M=%d,%s,momentum=%s,apply>" % (
+                         "frac": achieved / peak, "traffic": traffic, "traffic_source": traffic_note,
+                         "peak_source": peak_src,
+                         "frac_note": "the peak is a measured copy rate (1 read : 1 write), not a ceiling; "
+                                      "a stream with a larger share of reads can exceed it",
+                         "kernel": "%s<M=%d,%s,momentum=%s,apply>" % (
+                             "step_vec_kernel" if case.dtype == torch.float32 else "step_oct_bf16_kernel",
                              case.M, "f32" if case.dtype == torch.float32 else "bf16",
                              "yes" if case.beta is not None else "no"),
                          "algorithmic_bytes_per_launch": abytes,
                          "launch_ms": ms_step},
             "gpu_launches": args.steps,
             "clocks": clocks,
+            "ms_x_sm_mhz": ms_step * sm_mhz if sm_mhz else None,
         }
+        line.update(spread(per_launch))   # rank 0's own launches, one event pair each
+        line["per_launch"] = ("ms_median / ms_min / ms_max: a second pass of the same %d launches right after the "
+                              "timed region, an event after every launch; its total / steps = %.6f ms"
+                              % (args.steps, ms_again / args.steps))
+        line["ms_per_step_second_pass"] = ms_again / args.steps
         if e2e is not None:
             line["e2e"] = e2e
         if world == 1 and not args.no_cpu_baseline:
@@ -602,6 +694,152 @@ def main() -> None:
 
     if world > 1:
         dist.destroy_process_group()
+
+
+def worker_per_gpu_mode(args) -> None:
+    """--mode worker-per-gpu: Algorithm 1 with one worker per GPU (M = number of ranks). Every rank
+    owns one gradient buffer, its momentum and a replica of x; a step is MajorityVoteWorker.step:
+    momentum + sign packing of the local gradient, the exchange of packed signs in the chosen layout,
+    vote and parameter update. Prints ms per step, params/s, the bytes each worker receives per step
+    beside Appendix B's count, and the split of a step into kernel time and exchange time."""
+    import torch
+    import torch.distributed as dist
+
+    from paper_1810_05291_b200 import binding as B
+    from paper_1810_05291_b200 import inputs, sharding
+    from paper_1810_05291_b200.distributed import MajorityVoteWorker
+
+    world, rank, local_rank, dev = init_ranks()
+    if world == 1 and not dist.is_initialized():      # one-rank NCCL group: the real collectives, alone
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        os.environ.setdefault("MASTER_PORT", str(free_port()))
+        dist.init_process_group("nccl", rank=0, world_size=1, device_id=dev)
+    B.lib()
+    case = make_case(args.workload, args.d)
+    if case.beta is None and args.layout == "push":
+        raise SystemExit("the push layout carries the momentum kernel: use a workload with momentum")
+    case.M = world
+    stream = torch.cuda.current_stream()
+    s = inputs.signal(case, dev, 0)
+    grad = inputs.worker_gradient(case, rank, dev, 0, s)     # this worker's mini-batch gradient
+    del s
+    x = inputs.initial_params(case, dev)                     # same seed on every rank: one replica each
+    marks = []
+
+    def on_phase(label):
+        e = torch.cuda.Event(enable_timing=True)
+        e.record(stream)
+        marks.append((label, e))
+
+    worker = MajorityVoteWorker(x, case.beta, case.lr, case.weight_decay, args.layout, on_phase=on_phase)
+    if args.layout == "push":
+        worker.connect_push(barrier=args.push_barrier)
+
+    def step():
+        worker.step(grad, case.flip_mask & ((1 << world) - 1))
+
+    def barrier():
+        dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(args.warmup):
+        step()
+    barrier()
+    del marks[:]
+    ms_total, per_step, _, _ = timed_launches(step, args.steps, stream, barrier, per_launch=True)
+    # split: time between consecutive marks of a step goes to the phase that the later mark names
+    kernel_ms = exchange_ms = 0.0
+    phases = {}
+    for (la, ea), (lb, eb) in zip(marks, marks[1:]):
+        if lb == "start":
+            continue
+        dt = ea.elapsed_time(eb)
+        phases[lb] = phases.get(lb, 0.0) + dt
+        if lb.startswith("kernel:"):
+            kernel_ms += dt
+        else:
+            exchange_ms += dt
+    launches_per_step = sum(1 for (l, _) in marks if l.startswith("kernel:")) // max(1, args.steps)
+    ms_total = sharding.max_over_ranks(ms_total, dev)
+    kernel_ms = sharding.max_over_ranks(kernel_ms, dev)
+    exchange_ms = sharding.max_over_ranks(exchange_ms, dev)
+    ms_step = ms_total / args.steps
+    if rank == 0:
+        W4 = ((case.d + 31) // 32) * 4
+        paper_bits = 2 * world * case.d                      # Appendix B: 2 M d bits per iteration, whole system
+        line = {
+            "mode": "worker-per-gpu", "layout": args.layout, "metric": "majority-vote step params/s",
+            "value": case.d / (ms_step * 1e-3), "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "strong",
+            "dtype": dtype_name(case), "data": "synthetic",
+            "config": {"workload": case.name, "M": world, "d": case.d, "beta": case.beta, "lr": case.lr,
+                       "layout": args.layout,
+                       "push_barrier": args.push_barrier if args.layout == "push" else None},
+            "kernel_ms_per_step": kernel_ms / args.steps, "exchange_ms_per_step": exchange_ms / args.steps,
+            "phases_ms_per_step": {k: v / args.steps for k, v in sorted(phases.items())},
+            "bytes_received_per_worker_per_step": worker.ex.bytes_received_per_step(),
+            "bytes_received_allgather_formula": (world - 1) * W4,
+            "bytes_received_sharded_formula": 2 * (world - 1) * W4 // world,
+            "paper_bits_per_iteration_whole_system": paper_bits,
+            "gpu_launches": launches_per_step * args.steps,
+            "note": ("M = number of ranks: every rank is one worker of Algorithm 1 with its own replica of x; "
+                     "params/s counts the d parameters once"),
+        }
+        line.update(spread(per_step))
+        print(json.dumps(line), flush=True)
+    dist.destroy_process_group()
+
+
+def main() -> None:
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="cfg3")
+    ap.add_argument("--d", "--coords", dest="d", type=int, default=None,
+                    help="override the coordinate count (tests, profiling); --coords is the spelling to use "
+                         "under torchrun, whose own parser finds --d ambiguous")
+    ap.add_argument("--mode", default="fused", choices=["fused", "worker-per-gpu", "launch-check"],
+                    help="fused: ss_fused_step on every rank's coordinate shard (the headline number); "
+                         "worker-per-gpu: one worker of Algorithm 1 per GPU with the packed-sign exchange; "
+                         "launch-check: CPU-only check of the multi-rank launcher")
+    ap.add_argument("--layout", default="allgather", choices=["allgather", "sharded", "push"],
+                    help="worker-per-gpu: how the packed signs are exchanged")
+    ap.add_argument("--push-barrier", default="collective", choices=["collective", "signal"],
+                    help="worker-per-gpu, push layout: barrier between the push and the reads")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--profile", action="store_true",
+                    help="for runs under a profiler: no clock sampling, no end-to-end and CPU legs")
+    ap.add_argument("--table", default=None,
+                    help="time every entry point: 'named' (cfg1-4), 'sweep' (the d x M sweep) or a "
+                         "comma-separated list of workloads; one JSON line per row, then a table")
+    ap.add_argument("--entries", default=None,
+                    help="with --table: comma-separated entry points to time instead of the table's own list")
+    ap.add_argument("--threads", type=int, default=0, help="launch-shape override: block size")
+    ap.add_argument("--blocks-per-sm", type=int, default=0, help="launch-shape override")
+    args = ap.parse_args()
+    if args.warmup < 3:
+        args.warmup = 3
+    if args.profile:
+        args.no_e2e = args.no_cpu_baseline = True
+
+    if args.impl == "reference":
+        reference_arm(args)
+        return
+    if args.table:
+        table_mode(args)
+        return
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        # started as a plain process: become N ranks, one GPU each
+        sys.exit(spawn_ranks(args.gpus, sys.argv[1:]))
+    if args.mode == "launch-check":
+        launch_check_mode(args)
+    elif args.mode == "worker-per-gpu":
+        worker_per_gpu_mode(args)
+    else:
+        fused_mode(args)
 
 
 if __name__ == "__main__":

@@ -16,10 +16,10 @@ this GPU's own memory before a kernel reads them.
 
 ``push``       the all-gather folded into the producing kernel: ``ss_signum_update_push`` stores
                each packed word straight into this worker's slot of every worker's receive
-               buffer (peer stores over NVLink), a barrier across the workers follows, and
-               ``ss_vote_apply`` reads the local receive buffer. The caller supplies the peer
-               addresses (``set_push_destinations``) and the barrier. Signum only. Not run on
-               more than one GPU here: on one GPU the destinations are local buffers.
+               buffer (plain peer stores over NVLink), a barrier across the workers follows, and
+               ``ss_vote_apply`` reads the local receive buffer. ``connect_push`` sets up the
+               peer addresses and the barrier (by default a one-element all-reduce in stream
+               order); ``set_push_destinations`` takes them from the caller. Signum only.
 
 ``PackedExchange`` holds the buffers and the slice arithmetic and works on any device (the
 multi-process CPU tests drive it over gloo); ``MajorityVoteWorker`` adds the kernels and needs
@@ -113,16 +113,24 @@ class PackedExchange:
 
 class MajorityVoteWorker:
     """Algorithm 1 as seen from one worker: momentum and sign packing of the local gradient,
-    the exchange, then vote and parameter update. State (x, v) lives on this worker's GPU."""
+    the exchange, then vote and parameter update. State (x, v) lives on this worker's GPU.
+
+    ``kernels`` is the object whose ``ss_*`` functions do the arithmetic: by default the binding
+    of the CUDA library (tensors must then be CUDA tensors; there is no CPU path). The host-side
+    tests pass a stand-in so that the order of kernels and collectives can be driven on CPU ranks.
+    ``on_phase`` (optional) is called with a label after every kernel or collective of a step has
+    been enqueued -- the benchmark records a CUDA event there to split a step into kernel time
+    and exchange time."""
 
     def __init__(self, param: torch.Tensor, beta: Optional[float], lr: float,
                  weight_decay: float = 0.0, mode: str = "allgather", group=None, world=None,
-                 rank=None, collectives=None):
-        from . import binding as B
-        if not param.is_cuda:
-            raise ValueError("MajorityVoteWorker needs CUDA tensors: the arithmetic has no CPU path")
-        B.lib()
-        self.B = B
+                 rank=None, collectives=None, kernels=None, on_phase=None):
+        if kernels is None:
+            from . import binding as kernels
+            if not param.is_cuda:
+                raise ValueError("MajorityVoteWorker needs CUDA tensors: the arithmetic has no CPU path")
+            kernels.lib()
+        self.B = kernels
         self.x = param
         self.d = param.numel()
         self.beta, self.lr, self.weight_decay = beta, float(lr), float(weight_decay)
@@ -135,29 +143,43 @@ class MajorityVoteWorker:
         self.vote = torch.zeros(self.ex.W, dtype=torch.int32, device=param.device)
         self.push_dests = None
         self.barrier = None
+        self.on_phase = on_phase
         if mode == "push" and beta is None:
             raise ValueError("push mode carries the momentum kernel: use it with Signum (beta set)")
+
+    def _phase(self, label: str) -> None:
+        if self.on_phase is not None:
+            self.on_phase(label)
 
     def set_push_destinations(self, dests, barrier) -> None:
         """push mode: ``dests[m]`` is the address (tensor or int) of this worker's slot in worker
         m's receive buffer; ``barrier()`` must return only when every worker's push kernel has
-        completed, and is called again after the update so that no worker's next push overtakes
-        another worker's reads."""
+        completed (or, if it is stream-ordered, must order everything enqueued after it behind
+        every worker's push kernel), and is called again after the update so that no worker's next
+        push overtakes another worker's reads."""
         if len(dests) != self.ex.world:
             raise ValueError("need one destination per worker")
         self.push_dests = list(dests)
         self.barrier = barrier
 
-    def connect_push(self, group=None) -> None:
+    def connect_push(self, group=None, barrier: str = "collective") -> None:
         """push mode across GPUs: allocates the receive buffer in symmetric memory
         (``torch.distributed._symmetric_memory``), exchanges its addresses over ``group``, and
-        points this worker's push at its own slot in every peer's buffer. The barrier is the
-        handle's stream-ordered barrier, so push kernel, barrier, vote + update and second barrier
-        run in order on the current stream without host synchronisation. Every worker of the
-        group must call this once, after the process group exists."""
+        points this worker's push at its own slot in every peer's buffer. Every worker of the
+        group must call this once, after the process group exists.
+
+        ``barrier="collective"`` (default): the barrier between the push and the reads is a
+        one-element all-reduce of the process group (NCCL on GPUs), enqueued in stream order: it
+        starts when this worker's push kernel has finished and completes only when every worker
+        has reached it, and a worker that never arrives ends it with the process group's timeout
+        error on the host. ``barrier="signal"``: the symmetric-memory handle's own barrier, a
+        spin on a flag in the peers' signal pads inside a kernel, with the library's own timeout;
+        lower latency, kept as an explicit choice."""
         import torch.distributed._symmetric_memory as symm
         if self.ex.mode != "push":
             raise RuntimeError("connect_push is for push mode")
+        if barrier not in ("collective", "signal"):
+            raise ValueError("barrier must be 'collective' or 'signal'")
         group = group if group is not None else dist.group.WORLD
         ex = self.ex
         buf = symm.empty(ex.world * ex.W_pad, dtype=torch.int32, device=self.x.device)
@@ -167,7 +189,10 @@ class MajorityVoteWorker:
         slot_bytes = ex.W_pad * 4
         dests = [int(handle.buffer_ptrs[m]) + ex.rank * slot_bytes for m in range(ex.world)]
         self._symmetric = (buf, handle)
-        self.set_push_destinations(dests, handle.barrier)
+        if barrier == "signal":
+            self.set_push_destinations(dests, handle.barrier)
+        else:
+            self.set_push_destinations(dests, collective_barrier(group, self.x.device, ex.coll))
 
     def pack_local(self, grad: torch.Tensor, stream=None) -> None:
         """Worker side: v <- (1 - beta) g + beta v, sign(v) packed into the send buffer."""
@@ -179,17 +204,20 @@ class MajorityVoteWorker:
             self.B.ss_signum_update(grad, self.momentum, self.beta, self.ex.local_words(), stream)
         else:
             self.B.ss_sign_pack(grad, self.ex.local_words(), stream)
+        self._phase("kernel:pack")
 
     def serve(self, flip_mask: int = 0, stream=None) -> None:
         """sharded mode: receive every worker's words of this worker's slice and vote on them
-        (this worker acting as the parameter server of its slice). No-op in allgather mode."""
+        (this worker acting as the parameter server of its slice). No-op in the other modes."""
         ex = self.ex
         if ex.mode != "sharded":
             return
         ex.scatter_slices()
+        self._phase("exchange:all_to_all")
         n = ex.slice_coordinates()
         if n > 0:
             self.B.ss_majority_vote(ex.slice_rows(), n, flip_mask, ex.slice_vote(), stream)
+        self._phase("kernel:vote")
 
     def finish(self, flip_mask: int = 0, stream=None) -> torch.Tensor:
         """Receive what the update needs (all packed vectors, or the voted slices), update the
@@ -197,22 +225,43 @@ class MajorityVoteWorker:
         B, ex = self.B, self.ex
         if ex.mode == "push":
             self.barrier()
+            self._phase("exchange:barrier")
             B.ss_vote_apply(ex.worker_rows(), self.x, self.lr, self.weight_decay, flip_mask,
                             self.vote, stream)
+            self._phase("kernel:vote_apply")
             self.barrier()
+            self._phase("exchange:barrier")
             return self.vote
         if ex.mode == "allgather":
             ex.gather()
+            self._phase("exchange:all_gather")
             B.ss_vote_apply(ex.worker_rows(), self.x, self.lr, self.weight_decay, flip_mask,
                             self.vote, stream)
+            self._phase("kernel:vote_apply")
             return self.vote
         ex.gather_vote()
+        self._phase("exchange:all_gather")
         B.ss_apply_vote(self.x, ex.vote_words(), self.lr, self.weight_decay, stream)
+        self._phase("kernel:apply")
         return ex.vote_words()
 
     def step(self, grad: torch.Tensor, flip_mask: int = 0, stream=None) -> torch.Tensor:
         """One iteration. Kernels run on the current stream (or ``stream``, which must then be
         the stream the collectives see as current)."""
+        self._phase("start")
         self.pack_local(grad, stream)
         self.serve(flip_mask, stream)
         return self.finish(flip_mask, stream)
+
+
+def collective_barrier(group, device, collectives=None):
+    """A barrier made of a one-element all-reduce over ``group``: stream-ordered on GPUs (NCCL
+    enqueues it behind the work already on the current stream and the stream waits for it), and
+    bounded by the process group's timeout rather than by a device-side spin."""
+    coll = collectives if collectives is not None else dist
+    token = torch.zeros(1, dtype=torch.int32, device=device)
+
+    def barrier() -> None:
+        coll.all_reduce(token, group=group)
+
+    return barrier

@@ -16,7 +16,8 @@ import torch.distributed as dist
 import torch.multiprocessing as mp
 
 import oracle
-from paper_1810_05291_b200.distributed import PackedExchange, packed_words
+from paper_1810_05291_b200.distributed import (MajorityVoteWorker, PackedExchange, collective_barrier,
+                                               packed_words)
 
 
 def _free_port():
@@ -84,6 +85,116 @@ def _rank_main(rank, world, port, d, mode, flip):
     ("sharded", 2, 100_003, 0b01)])
 def test_workers_over_gloo_reproduce_the_m_worker_step(world, d, flip, mode):
     mp.spawn(_rank_main, args=(world, _free_port(), d, mode, flip), nprocs=world, join=True)
+
+
+class OracleKernels:
+    """Stand-in for the CUDA binding on CPU ranks: the same ``ss_*`` names and in-place behaviour,
+    served by the CPU oracle on views of the torch tensors. Only the tests use it; it lets
+    ``MajorityVoteWorker.step`` run unchanged, so that what is exercised is the order of kernels
+    and collectives and the buffers they are handed."""
+
+    def __init__(self):
+        self.calls = []
+
+    @staticmethod
+    def _f32(t):
+        return t.numpy()
+
+    @staticmethod
+    def _u32(t):
+        return t.numpy().view(np.uint32)
+
+    def ss_sign_pack(self, grad, out_words, stream=None):
+        self.calls.append("ss_sign_pack")
+        self._u32(out_words)[:] = oracle.sign_pack(self._f32(grad))
+
+    def ss_signum_update(self, grad, momentum, beta, out_words, stream=None):
+        self.calls.append("ss_signum_update")
+        self._u32(out_words)[:] = oracle.signum_update(self._f32(grad), self._f32(momentum), beta)
+
+    def ss_signum_update_push(self, grad, momentum, beta, dests, stream=None):
+        self.calls.append("ss_signum_update_push")
+        words = oracle.signum_update(self._f32(grad), self._f32(momentum), beta)
+        for dst in dests:
+            self._u32(dst)[:] = words
+
+    def ss_majority_vote(self, packed, d, flip_mask, vote_words, stream=None):
+        self.calls.append("ss_majority_vote")
+        self._u32(vote_words)[:] = oracle.majority_vote([self._u32(p).copy() for p in packed], d, flip_mask)
+
+    def ss_apply_vote(self, param, vote_words, lr, weight_decay=0.0, stream=None):
+        self.calls.append("ss_apply_vote")
+        oracle.apply_vote(self._f32(param), self._u32(vote_words).copy(), lr, weight_decay)
+
+    def ss_vote_apply(self, packed, param, lr, weight_decay=0.0, flip_mask=0, vote_words_out=None, stream=None):
+        self.calls.append("ss_vote_apply")
+        vote = oracle.majority_vote([self._u32(p).copy() for p in packed], param.numel(), flip_mask)
+        oracle.apply_vote(self._f32(param), vote, lr, weight_decay)
+        if vote_words_out is not None:
+            self._u32(vote_words_out)[:] = vote
+
+
+EXPECTED_ORDER = {
+    "allgather": ["start", "kernel:pack", "exchange:all_gather", "kernel:vote_apply"],
+    "sharded": ["start", "kernel:pack", "exchange:all_to_all", "kernel:vote", "exchange:all_gather",
+                "kernel:apply"],
+    "push": ["start", "kernel:pack", "exchange:barrier", "kernel:vote_apply", "exchange:barrier"],
+}
+
+
+def _worker_main(rank, world, port, d, mode, flip, beta, shared):
+    """One rank = one MajorityVoteWorker driven through step(); the oracle serves as its kernels."""
+    os.environ["MASTER_ADDR"] = "127.0.0.1"
+    os.environ["MASTER_PORT"] = str(port)
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    try:
+        lr, wd = 1e-3, 0.01
+        rng = np.random.default_rng(4321 + d)
+        x0 = rng.standard_normal(d).astype(np.float32)
+        phases = []
+        kernels = OracleKernels()
+        w = MajorityVoteWorker(torch.from_numpy(x0.copy()), beta, lr, wd, mode, world=world, rank=rank,
+                               kernels=kernels, on_phase=phases.append)
+        if mode == "push":
+            # the receive buffers live in shared memory: a stand-in for peer-mapped device memory,
+            # written by the other ranks' processes and ordered only by the barrier
+            w.ex.gathered = shared[rank]
+            slot = lambda buf: buf[rank * w.ex.W_pad: rank * w.ex.W_pad + w.ex.W]
+            w.set_push_destinations([slot(shared[m]) for m in range(world)],
+                                    collective_barrier(None, "cpu"))
+        ref_x = x0.copy()
+        ref_v = [np.zeros(d, dtype=np.float32) for _ in range(world)] if beta is not None else None
+        for step in range(3):
+            grads = [rng.standard_normal(d).astype(np.float32) for _ in range(world)]
+            want = oracle.fused_step(grads, ref_v, ref_x, beta if beta is not None else 0.0, lr, wd, flip)
+            del phases[:]
+            vote = w.step(torch.from_numpy(grads[rank].copy()), flip)
+            assert phases == EXPECTED_ORDER[mode], phases
+            assert np.array_equal(_as_u32(vote), want), "rank %d step %d: vote differs" % (rank, step)
+            assert np.array_equal(w.x.numpy().view(np.uint32), ref_x.view(np.uint32)), "rank %d: x differs" % rank
+            if beta is not None:
+                assert np.array_equal(w.momentum.numpy().view(np.uint32), ref_v[rank].view(np.uint32))
+        want_calls = {"allgather": ["ss_signum_update" if beta is not None else "ss_sign_pack", "ss_vote_apply"],
+                      "sharded": ["ss_signum_update" if beta is not None else "ss_sign_pack",
+                                  "ss_majority_vote", "ss_apply_vote"],
+                      "push": ["ss_signum_update_push", "ss_vote_apply"]}[mode]
+        if mode == "sharded" and w.ex.slice_coordinates() == 0:
+            want_calls = [c for c in want_calls if c != "ss_majority_vote"]
+        assert kernels.calls == want_calls * 3, kernels.calls
+    finally:
+        dist.destroy_process_group()
+
+
+@pytest.mark.parametrize("mode,world,d,flip,beta", [
+    ("allgather", 2, 100_003, 0b01, 0.9), ("allgather", 3, 70, 0, None),
+    ("sharded", 2, 1000, 0, 0.9), ("sharded", 3, 33, 0b010, None), ("sharded", 3, 100_003, 0b100, 0.9),
+    ("push", 2, 100_003, 0b10, 0.9), ("push", 3, 1000, 0, 0.9)])
+def test_majority_vote_worker_step_over_gloo(mode, world, d, flip, beta):
+    shared = None
+    if mode == "push":
+        W_pad = PackedExchange(d, world, 0, "meta", "push").W_pad
+        shared = [torch.zeros(world * W_pad, dtype=torch.int32).share_memory_() for _ in range(world)]
+    mp.spawn(_worker_main, args=(world, _free_port(), d, mode, flip, beta, shared), nprocs=world, join=True)
 
 
 @pytest.mark.parametrize("d,world", [(1, 1), (1, 4), (31, 2), (32, 2), (33, 2), (1000, 3), (1024, 4),

@@ -1,11 +1,13 @@
-"""MajorityVoteWorker on one GPU.
+"""MajorityVoteWorker on GPUs.
 
-Only one GPU is available to these tests, so the M workers of Algorithm 1 are M worker objects
-in one process whose collectives are served by an in-process stand-in that copies between their
-buffers (all on one stream, one after another: no kernel waits on another). The kernels, the
-buffers and the slice arithmetic are the ones a multi-GPU run uses; the NCCL transport itself is
-exercised with a one-rank process group. Every worker must end each step with the parameters,
-momentum and packed vote of the oracle's M-worker step.
+On one GPU the M workers of Algorithm 1 are M worker objects in one process whose collectives are
+served by an in-process stand-in that copies between their buffers (all on one stream, one after
+another: no kernel waits on another). The kernels, the buffers and the slice arithmetic are the
+ones a multi-GPU run uses; the NCCL transport itself is exercised with a one-rank process group.
+Where the machine has two or three GPUs, the last test runs one worker per GPU as separate
+processes over NCCL in all three exchange layouts; with fewer GPUs it is reported as skipped (a
+skip proves nothing about that path). Every worker must end each step with the parameters, momentum
+and packed vote of the oracle's M-worker step.
 """
 import os
 import socket
@@ -128,10 +130,12 @@ def test_one_rank_nccl_group_runs_the_real_collectives(mode):
         dist.destroy_process_group()
 
 
-def test_push_mode_over_symmetric_memory_with_one_rank():
+@pytest.mark.parametrize("barrier", ["collective", "signal"])
+def test_push_mode_over_symmetric_memory_with_one_rank(barrier):
     """The symmetric-memory wiring of push mode on a one-rank group: the receive buffer is a
-    symmetric allocation, the push goes to the address the rendezvous reports, and the handle's
-    barrier orders the steps. (More ranks need more GPUs than these tests have.)"""
+    symmetric allocation, the push goes to the address the rendezvous reports, and the barrier (a
+    stream-ordered one-element all-reduce by default, the handle's signal barrier on request)
+    orders the steps."""
     with socket.socket() as s:
         s.bind(("127.0.0.1", 0))
         port = s.getsockname()[1]
@@ -145,7 +149,7 @@ def test_push_mode_over_symmetric_memory_with_one_rank():
         x0 = rng.standard_normal(d).astype(np.float32)
         w = MajorityVoteWorker(torch.from_numpy(x0.copy()).to(DEV), 0.9, 1e-3, 0.0, "push")
         try:
-            w.connect_push()
+            w.connect_push(barrier=barrier)
         except (RuntimeError, NotImplementedError) as e:
             pytest.skip("symmetric memory is not available here: %s" % str(e)[:200])
         ref_x, ref_v = x0.copy(), [np.zeros(d, dtype=np.float32)]
@@ -158,3 +162,54 @@ def test_push_mode_over_symmetric_memory_with_one_rank():
             assert np.array_equal(w.x.cpu().numpy().view(np.uint32), ref_x.view(np.uint32))
     finally:
         dist.destroy_process_group()
+
+
+def _nccl_worker(rank, world, port, mode, d, beta, flip, errors):
+    """One process = one worker of Algorithm 1 on GPU `rank`, talking NCCL to the others."""
+    os.environ["MASTER_ADDR"] = "127.0.0.1"
+    os.environ["MASTER_PORT"] = str(port)
+    os.environ["NCCL_NVLS_ENABLE"] = "0"          # plain peer traffic only
+    try:
+        torch.cuda.set_device(rank)
+        dev = torch.device("cuda", rank)
+        dist.init_process_group("nccl", rank=rank, world_size=world, device_id=dev)
+        try:
+            rng = np.random.default_rng(5000 + d + world)
+            x0 = rng.standard_normal(d).astype(np.float32)
+            w = MajorityVoteWorker(torch.from_numpy(x0.copy()).to(dev), beta, 1e-3, 0.01, mode)
+            if mode == "push":
+                w.connect_push()
+            ref_x = x0.copy()
+            ref_v = [np.zeros(d, dtype=np.float32) for _ in range(world)] if beta is not None else None
+            for step in range(4):
+                grads = [rng.standard_normal(d).astype(np.float32) for _ in range(world)]
+                want = oracle.fused_step(grads, ref_v, ref_x, beta if beta is not None else 0.0, 1e-3, 0.01, flip)
+                vote = w.step(torch.from_numpy(grads[rank]).to(dev), flip)
+                torch.cuda.synchronize()
+                assert np.array_equal(vote.cpu().numpy().view(np.uint32), want), "vote, step %d" % step
+                assert np.array_equal(w.x.cpu().numpy().view(np.uint32), ref_x.view(np.uint32)), "x, step %d" % step
+                if beta is not None:
+                    assert np.array_equal(w.momentum.cpu().numpy().view(np.uint32), ref_v[rank].view(np.uint32))
+        finally:
+            dist.destroy_process_group()
+    except Exception as e:                          # reported by the parent
+        errors.put("rank %d: %r" % (rank, e))
+        raise
+
+
+@pytest.mark.parametrize("world", [2, 3])
+@pytest.mark.parametrize("mode,beta", [("allgather", 0.9), ("allgather", None), ("sharded", 0.9), ("push", 0.9)])
+def test_one_worker_per_gpu_over_nccl(world, mode, beta):
+    if torch.cuda.device_count() < world:
+        pytest.skip("needs %d GPUs, this machine shows %d: the one-worker-per-GPU path over NCCL is "
+                    "not exercised here" % (world, torch.cuda.device_count()))
+    import torch.multiprocessing as mp
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        port = s.getsockname()[1]
+    ctx = mp.get_context("spawn")
+    errors = ctx.Queue()
+    d = 32 * 40_000 + 8
+    flip = 0b10
+    mp.spawn(_nccl_worker, args=(world, port, mode, d, beta, flip, errors), nprocs=world, join=True)
+    assert errors.empty()
