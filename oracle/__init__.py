@@ -22,6 +22,7 @@ import numpy as np
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
 _SRC = os.path.join(_HERE, "signsgd_oracle.cpp")
+_SRC_TERNARY = os.path.join(_HERE, "ternary_oracle.cpp")   # the comparison codec of Appendix B
 _LIB = os.path.join(_HERE, "libsignsgd_oracle.so")
 _lock = threading.Lock()
 _lib = None
@@ -34,11 +35,11 @@ def build(force: bool = False) -> str:
     """Compile the oracle with g++ (-O2 -ffp-contract=off: no fused multiply-add, so the
     momentum is two rounded multiplies and one rounded add as Algorithm 1's line is read)."""
     if (not force and os.path.exists(_LIB)
-            and os.path.getmtime(_LIB) >= os.path.getmtime(_SRC)):
+            and os.path.getmtime(_LIB) >= max(os.path.getmtime(_SRC), os.path.getmtime(_SRC_TERNARY))):
         return _LIB
     tmp = _LIB + ".tmp.%d" % os.getpid()
     cmd = ["g++", "-std=c++17", "-O2", "-ffp-contract=off", "-fno-fast-math", "-fopenmp",
-           "-fPIC", "-shared", "-o", tmp, _SRC]
+           "-fPIC", "-shared", "-o", tmp, _SRC, _SRC_TERNARY]
     subprocess.run(cmd, check=True)
     os.replace(tmp, _LIB)
     return _LIB
@@ -70,6 +71,18 @@ def _load():
         lib.oracle_apply_vote.restype = None
         lib.oracle_fused_step.argtypes = [vp, i32, vp, i32, i64, f32, u64, vp, f32, f32, vp]
         lib.oracle_fused_step.restype = None
+        lib.oracle_philox4x32_10.argtypes = [vp, vp, vp]
+        lib.oracle_philox4x32_10.restype = None
+        lib.oracle_ternary_draws.argtypes = [u64, i64, vp]
+        lib.oracle_ternary_draws.restype = None
+        lib.oracle_absmax.argtypes = [vp, i32, i64]
+        lib.oracle_absmax.restype = f32
+        lib.oracle_ternary_words.argtypes = [i64]
+        lib.oracle_ternary_words.restype = i64
+        lib.oracle_ternary_pack.argtypes = [vp, i32, i64, f32, vp, vp]
+        lib.oracle_ternary_pack.restype = None
+        lib.oracle_ternary_unpack.argtypes = [vp, i64, f32, vp]
+        lib.oracle_ternary_unpack.restype = None
         _lib = lib
         return lib
 
@@ -208,3 +221,57 @@ def fused_step_segments(grads, momenta, param: np.ndarray, beta: float, begins, 
                    [v[a:b] for v in momenta] if momenta is not None else None,
                    param[a:b], beta, float(lrs[k]), float(weight_decays[k]), flip_mask)
     return vote
+
+
+# ---- the comparison codec of Appendix B: 1-bit max-norm QSGD (ternary, two bits per coordinate) ----
+
+def philox4x32_10(counter, key) -> np.ndarray:
+    """One block of the counter-based generator: 4 counter words, 2 key words -> 4 output words."""
+    c = np.asarray(counter, dtype=np.uint32).copy()
+    k = np.asarray(key, dtype=np.uint32).copy()
+    if c.shape != (4,) or k.shape != (2,):
+        raise ValueError("counter has 4 words, key has 2")
+    out = np.zeros(4, dtype=np.uint32)
+    _load().oracle_philox4x32_10(_ptr(c), _ptr(k), _ptr(out))
+    return out
+
+
+def ternary_draws(seed: int, d: int) -> np.ndarray:
+    """The 32-bit draw of every coordinate 0..d-1 under a seed."""
+    r = np.zeros(int(d), dtype=np.uint32)
+    _load().oracle_ternary_draws(int(seed), int(d), _ptr(r))
+    return r
+
+
+def absmax(grad: np.ndarray) -> float:
+    """||g||_inf over the elements that are not NaN, as fp32."""
+    dt = _grad(grad)
+    return float(_load().oracle_absmax(_ptr(grad), dt, grad.shape[0]))
+
+
+def ternary_words(d: int) -> int:
+    return int(_load().oracle_ternary_words(int(d)))
+
+
+def ternary_pack(grad: np.ndarray, gmax: float = None, seed: int = None, draws: np.ndarray = None) -> np.ndarray:
+    """1-bit max-norm QSGD code of a gradient: two bits per coordinate, 16 per uint32 word. The
+    draws are either given (one uint32 per coordinate) or generated from ``seed``."""
+    dt = _grad(grad)
+    d = grad.shape[0]
+    if gmax is None:
+        gmax = absmax(grad)
+    if draws is None:
+        if seed is None:
+            raise ValueError("give either the draws or a seed")
+        draws = ternary_draws(seed, d)
+    _check(draws, np.uint32, d, "draws")
+    codes = np.zeros(ternary_words(d), dtype=np.uint32)
+    _load().oracle_ternary_pack(_ptr(grad), dt, d, float(np.float32(gmax)), _ptr(draws), _ptr(codes))
+    return codes
+
+
+def ternary_unpack(codes: np.ndarray, d: int, scale: float) -> np.ndarray:
+    _check(codes, np.uint32, ternary_words(d), "codes")
+    out = np.zeros(int(d), dtype=np.float32)
+    _load().oracle_ternary_unpack(_ptr(codes), int(d), float(np.float32(scale)), _ptr(out))
+    return out
