@@ -291,6 +291,13 @@ def entry_bytes(case, entry: str) -> int:
         return M * wb + 8 * d
     if entry in ("fused", "fused_segments"):
         return algorithmic_bytes(case)
+    tb = ((d + 15) // 16) * 4            # the ternary comparison codec: 2 bits per coordinate
+    if entry == "absmax":
+        return gb * d
+    if entry == "ternary_pack":
+        return gb * d + tb
+    if entry == "ternary_unpack":
+        return tb + 4 * d
     if entry == "chain":
         per_worker = entry_bytes(case, "signum_update" if mom else "pack")
         return M * per_worker + entry_bytes(case, "vote") + entry_bytes(case, "apply")
@@ -381,10 +388,21 @@ def table_mode(args) -> None:
         seg_table = B.segment_table(n_seg, dev)
         B.ss_segments_upload(seg_begins, [case.lr] * n_seg, [case.weight_decay] * n_seg, case.d, seg_table, stream)
 
+        gmax = torch.zeros(1, device=dev)
+        codes = torch.zeros(B.ss_ternary_words(case.d), dtype=torch.int32, device=dev)
+        decoded = torch.empty(case.d, device=dev) if args.entries and "ternary_unpack" in entries else None
+        B.ss_absmax(grads[0], gmax, stream)
+
         def call(entry):
             m = turn[0] % case.M
             turn[0] += 1
-            if entry == "pack":
+            if entry == "absmax":
+                B.ss_absmax(grads[m], gmax, stream)
+            elif entry == "ternary_pack":
+                B.ss_ternary_pack(grads[m], gmax, 1000 + turn[0], codes, stream)
+            elif entry == "ternary_unpack":
+                B.ss_ternary_unpack(codes, gmax, decoded, stream)
+            elif entry == "pack":
                 B.ss_sign_pack(grads[m], packed[m], stream)
             elif entry == "signum_update":
                 B.ss_signum_update(grads[m], moms[m], beta, packed[m], stream)

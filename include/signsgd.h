@@ -279,6 +279,51 @@ int ss_fused_step_host_static(const void* const* host_grads, ss_dtype dt, float*
                               uint32_t* host_vote_out, void* cuda_stream);
 
 /*
+ * The comparison codec of Appendix B: 1-bit max-norm QSGD, the ternary quantiser against which
+ * the paper sets the bits per iteration of majority vote. Coordinate g_i becomes sign(g_i) with
+ * probability |g_i| / ||g||_inf and 0 otherwise; the code takes two bits per coordinate (Appendix
+ * B: 2d bits always store d numbers in {0, +-1}), 16 coordinates per uint32 word: coordinate
+ * 16 j + i sits at bits 2i, 2i+1 of word j as 0 (zero), 1 (+1) or 3 (-1); bits at coordinates
+ * >= d are 0. A comparison system, not a step of Algorithm 1.
+ *
+ * The draws come from the Philox4x32-10 counter-based generator evaluated inside the kernel:
+ * the block with counter (q, 0, 0) [q split into two 32-bit words] and key `seed` gives the four
+ * 32-bit words r of coordinates 4q .. 4q+3. With u = (r >> 9) * 2^-23, a coordinate is kept iff
+ * RN(u * ||g||_inf) < |g_i| in fp32: the maximum is always kept, zeros and NaNs never; nothing is
+ * kept when ||g||_inf is 0 or Inf. The same (gradient, max-norm, seed) always gives the same code.
+ */
+
+/* ceil(d/16): words of a ternary code. -1 if d < 0. */
+int64_t ss_ternary_words(int64_t d);
+
+/*
+ * ||g||_inf = max |g_i| over the elements that are not NaN (0 for d == 0), as fp32.
+ *   grad        in   d elements of dtype dt
+ *   absmax_dev  out  one fp32 in DEVICE memory (zeroed, then raised by the kernel)
+ */
+int ss_absmax(const void* grad, ss_dtype dt, int64_t d, float* absmax_dev, void* cuda_stream);
+
+/*
+ * Ternary code of one worker's gradient.
+ *   grad        in   d elements of dtype dt
+ *   absmax_dev  in   DEVICE pointer to ||g||_inf as written by ss_absmax on the same stream
+ *   seed        in   key of the generator; use a fresh one per worker and per step
+ *   out_codes   out  ceil(d/16) words
+ */
+int ss_ternary_pack(const void* grad, ss_dtype dt, int64_t d, const float* absmax_dev, uint64_t seed,
+                    uint32_t* out_codes, void* cuda_stream);
+
+/*
+ * Decoder: out_i = scale * q_i with q_i in {0, +-1} read from the code (QSGD's estimate of the
+ * gradient uses scale = ||g||_inf; its expectation over the draws is g).
+ *   codes      in   ceil(d/16) words
+ *   scale_dev  in   DEVICE pointer to one fp32
+ *   out        out  d fp32
+ */
+int ss_ternary_unpack(const uint32_t* codes, int64_t d, const float* scale_dev, float* out,
+                      void* cuda_stream);
+
+/*
  * Launch-shape override for benchmarking sweeps: not part of the method, and the one piece of
  * process-wide state in the library (two integers, written and read atomically; a launch uses the
  * values it finds when it is made, so change them only between calls whose shape matters).

@@ -8,10 +8,10 @@
 // Readings fixed here (Appendix B gives the probabilities, not an encoding or a generator):
 //   T1  ||g||_inf is the largest |g_i| over the elements that are not NaN (0 for an empty or
 //       all-NaN vector), in fp32.
-//   T2  The draw for coordinate c is a 32-bit word r_c; u_c = (r_c >> 8) * 2^-24 is uniform on the
-//       2^24 multiples of 2^-24 in [0, 1). The coordinate is kept iff RN(u_c * ||g||_inf) < |g_c|,
+//   T2  The draw for coordinate c is a 32-bit word r_c; u_c = (r_c >> 9) * 2^-23 is uniform on the
+//       2^23 multiples of 2^-23 in [0, 1). The coordinate is kept iff RN(u_c * ||g||_inf) < |g_c|,
 //       one rounded fp32 multiply and one comparison: probability |g_c| / ||g||_inf to within
-//       2^-24. |g_c| = ||g||_inf is always kept (so a sign vector comes through unchanged, as
+//       2^-23. |g_c| = ||g||_inf is always kept (so a sign vector comes through unchanged, as
 //       Appendix B notes), g_c = 0 never, NaN never; if ||g||_inf is Inf nothing is kept.
 //   T3  Code of coordinate c: 0 for zero, 1 for +1, 3 for -1 (low bit "kept", high bit
 //       "negative"), at bits 2i, 2i+1 of word j for c = 16 j + i; bits beyond d are 0.
@@ -107,7 +107,7 @@ void oracle_ternary_pack(const void* grad, int dtype, int64_t d, float gmax, con
     for (int64_t j = 0; j < oracle_ternary_words(d); ++j) codes[j] = 0u;
     for (int64_t c = 0; c < d; ++c) {
         const float g = grad_at(grad, dtype, c);
-        const float u = static_cast<float>(r[c] >> 8) * 5.9604644775390625e-08f;  // exact: 24 bits * 2^-24
+        const float u = static_cast<float>(r[c] >> 9) * 1.1920928955078125e-07f;  // exact: 23 bits * 2^-23
         const float t = u * gmax;                                                // one rounded multiply
         const bool kept = t < std::fabs(g);                                      // false for NaN
         uint32_t code = 0u;

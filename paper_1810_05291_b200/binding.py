@@ -35,7 +35,8 @@ SS_ERR_CUDA = -4
 EXPORTS = ("ss_packed_words", "ss_status_string", "ss_last_cuda_error", "ss_sign_pack",
            "ss_majority_vote", "ss_signum_update", "ss_apply_vote", "ss_fused_step",
            "ss_segments_upload", "ss_fused_step_segments", "ss_apply_vote_segments",
-           "ss_vote_apply", "ss_vote_apply_segments", "ss_signum_update_push", "ss_vote_tally", "ss_fused_step_host", "ss_fused_step_host_static", "ss_set_launch_option")
+           "ss_vote_apply", "ss_vote_apply_segments", "ss_signum_update_push", "ss_vote_tally", "ss_fused_step_host", "ss_fused_step_host_static", "ss_set_launch_option",
+           "ss_ternary_words", "ss_absmax", "ss_ternary_pack", "ss_ternary_unpack")
 
 
 class ss_segment(ctypes.Structure):
@@ -90,6 +91,13 @@ def lib() -> ctypes.CDLL:
     L.ss_vote_tally.argtypes = [vp, i32, i64, u64, vp, vp]
     L.ss_vote_apply.argtypes = [vp, i32, i64, u64, vp, f32, f32, vp, vp]
     L.ss_vote_apply_segments.argtypes = [vp, i32, i64, u64, vp, vp, i32, vp, vp]
+    L.ss_ternary_words.argtypes = [i64]
+    L.ss_ternary_words.restype = i64
+    L.ss_absmax.argtypes = [vp, i32, i64, vp, vp]
+    L.ss_ternary_pack.argtypes = [vp, i32, i64, vp, u64, vp, vp]
+    L.ss_ternary_unpack.argtypes = [vp, i64, vp, vp, vp]
+    for name in ("ss_absmax", "ss_ternary_pack", "ss_ternary_unpack"):
+        getattr(L, name).restype = i32
     for name in ("ss_sign_pack", "ss_majority_vote", "ss_signum_update", "ss_apply_vote",
                  "ss_fused_step", "ss_fused_step_host", "ss_fused_step_host_static",
                  "ss_set_launch_option", "ss_segments_upload", "ss_fused_step_segments",
@@ -373,3 +381,30 @@ def ss_fused_step_host_static(host_grads: Sequence[torch.Tensor],
                                            float(lr), float(weight_decay),
                                            _words(vote_words_dev, d, "vote_words_dev"), hv,
                                            _stream(stream)), "ss_fused_step_host_static")
+
+
+# ---- the comparison codec of Appendix B (1-bit max-norm QSGD) -------------------------------
+
+def ss_ternary_words(d: int) -> int:
+    return int(lib().ss_ternary_words(int(d)))
+
+
+def ss_absmax(grad: torch.Tensor, absmax_dev: torch.Tensor, stream=None) -> None:
+    _check(lib().ss_absmax(_dev(grad, None, "grad"), _dtype_code(grad), grad.numel(),
+                           _dev(absmax_dev, torch.float32, "absmax_dev", 1), _stream(stream)), "ss_absmax")
+
+
+def ss_ternary_pack(grad: torch.Tensor, absmax_dev: torch.Tensor, seed: int, out_codes: torch.Tensor,
+                    stream=None) -> None:
+    d = grad.numel()
+    _check(lib().ss_ternary_pack(_dev(grad, None, "grad"), _dtype_code(grad), d,
+                                 _dev(absmax_dev, torch.float32, "absmax_dev", 1), int(seed),
+                                 _dev(out_codes, torch.int32, "out_codes", ss_ternary_words(d)),
+                                 _stream(stream)), "ss_ternary_pack")
+
+
+def ss_ternary_unpack(codes: torch.Tensor, scale_dev: torch.Tensor, out: torch.Tensor, stream=None) -> None:
+    d = out.numel()
+    _check(lib().ss_ternary_unpack(_dev(codes, torch.int32, "codes", ss_ternary_words(d)), d,
+                                   _dev(scale_dev, torch.float32, "scale_dev", 1),
+                                   _dev(out, torch.float32, "out"), _stream(stream)), "ss_ternary_unpack")
