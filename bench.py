@@ -350,6 +350,10 @@ def table_mode(args) -> None:
     dev = torch.device("cuda", 0)
     torch.cuda.set_device(dev)
     B.lib()
+    if args.threads:
+        B.ss_set_launch_option("threads", args.threads)
+    if args.blocks_per_sm:
+        B.ss_set_launch_option("blocks_per_sm", args.blocks_per_sm)
     stream = torch.cuda.current_stream()
     flush = torch.empty(512 << 20, dtype=torch.uint8, device=dev)
     peak, peak_src = measured_peak()
@@ -777,7 +781,9 @@ def worker_per_gpu_mode(args) -> None:
             kernel_ms += dt
         else:
             exchange_ms += dt
-    launches_per_step = sum(1 for (l, _) in marks if l.startswith("kernel:")) // max(1, args.steps)
+    ours = ("kernel:", "exchange:signal", "exchange:wait")     # phases that are launches of this library's kernels
+    launches_per_step = sum(1 for (l, _) in marks if l.startswith(ours)) // max(1, args.steps)
+    worker.check()
     ms_total = sharding.max_over_ranks(ms_total, dev)
     kernel_ms = sharding.max_over_ranks(kernel_ms, dev)
     exchange_ms = sharding.max_over_ranks(exchange_ms, dev)
@@ -824,8 +830,10 @@ def main() -> None:
                          "launch-check: CPU-only check of the multi-rank launcher")
     ap.add_argument("--layout", default="allgather", choices=["allgather", "sharded", "push"],
                     help="worker-per-gpu: how the packed signs are exchanged")
-    ap.add_argument("--push-barrier", default="collective", choices=["collective", "signal"],
-                    help="worker-per-gpu, push layout: barrier between the push and the reads")
+    ap.add_argument("--push-barrier", default="collective", choices=["collective", "signal", "flags"],
+                    help="worker-per-gpu, push layout: what orders the push before the reads: a one-element "
+                         "all-reduce (collective), the symmetric-memory signal barrier (signal), or the library's "
+                         "own flags with a bounded wait and no collective at all (flags)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--profile", action="store_true",

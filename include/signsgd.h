@@ -159,6 +159,53 @@ int ss_vote_apply(const uint32_t* const* packed, int M, int64_t d, uint64_t flip
                   float lr, float weight_decay, uint32_t* vote_words_out, void* cuda_stream);
 
 /*
+ * Flag-ordered exchange for one worker per GPU (Algorithm 1's "push sign(v_m) to server" and
+ * "push sign(V) to each worker", with every worker acting as its own server). Each worker owns a
+ * flag array of SS_MAX_WORKERS uint32 words in its memory, mapped into its peers. A step with
+ * epoch e (1, 2, 3, ... ; serial-number comparison, so wrap-around is harmless):
+ *   1. ss_signum_update_push stores this worker's packed signs into its slot of every worker's
+ *      receive buffer;
+ *   2. ss_flags_signal, on the same stream, writes e into word `index` (= this worker's rank) of
+ *      every worker's flag array: it runs once the push kernel has completed, so a peer that sees
+ *      the flag sees the words;
+ *   3. ss_flags_wait polls this worker's OWN flag array until words 0 .. M-1 have all reached e,
+ *      for at most timeout_ns, and writes 0 or (1 + lowest missing worker) to *status_dev;
+ *   4. ss_vote_apply_guarded votes and updates unless *status_dev is non-zero, in which case the
+ *      whole launch does nothing: parameters are updated for all coordinates or for none.
+ * Two receive buffers used alternately (by the parity of e) make a second synchronisation
+ * unnecessary: a worker reaches its push of step e+2 only after its wait of step e+1, i.e. after
+ * every peer has finished its update of step e, which is what read the buffer now overwritten.
+ * Only plain stores go to a peer; nothing is read from one; the only wait is the bounded one of
+ * step 3, on local memory. The host decides what a time-out means: read *status_dev after
+ * synchronising the stream (a worker left, or is late), before trusting the step.
+ */
+#define SS_FLAGS_MAX_TIMEOUT_NS 2000000000ull /* 2 s: the longest wait ss_flags_wait accepts */
+
+/*   flags    in   HOST array of n_flags device pointers, each to a flag array (4-byte aligned)
+ *   index    in   word to write in each array, 0 .. SS_MAX_WORKERS-1 (the signalling worker's rank)
+ *   epoch    in   value to write */
+int ss_flags_signal(uint32_t* const* flags, int n_flags, int index, uint32_t epoch, void* cuda_stream);
+
+/*   flags_local  in   this worker's own flag array (device memory of the current device)
+ *   M            in   workers to wait for: words 0 .. M-1
+ *   timeout_ns   in   at most SS_FLAGS_MAX_TIMEOUT_NS, else SS_ERR_INVALID_ARG
+ *   status_dev   out  one uint32 in device memory: 0, or 1 + the lowest worker that did not arrive
+ * One block of SS_MAX_WORKERS threads; it always terminates (time limit, plus an iteration limit
+ * as a backstop) and leaves the context usable. */
+int ss_flags_wait(const uint32_t* flags_local, int M, uint32_t epoch, uint64_t timeout_ns,
+                  uint32_t* status_dev, void* cuda_stream);
+
+/* ss_flags_signal followed by ss_flags_wait in one launch (steps 2 and 3 above back to back). */
+int ss_flags_signal_wait(uint32_t* const* flags, int n_flags, int index, const uint32_t* flags_local, int M,
+                         uint32_t epoch, uint64_t timeout_ns, uint32_t* status_dev, void* cuda_stream);
+
+/* ss_vote_apply that does nothing at all when the word at skip_if_nonzero_dev (device memory,
+ * written by an earlier call on the same stream, e.g. ss_flags_wait) is not zero. */
+int ss_vote_apply_guarded(const uint32_t* const* packed, int M, int64_t d, uint64_t flip_mask,
+                          float* param, float lr, float weight_decay, uint32_t* vote_words_out,
+                          const uint32_t* skip_if_nonzero_dev, void* cuda_stream);
+
+/*
  * One whole iteration of Algorithm 1 in a single pass over memory: momentum, sign, vote and
  * parameter update per coordinate, the packed signs never leaving the chip.
  *   grads           in      HOST array of M device pointers, d elements of dt each

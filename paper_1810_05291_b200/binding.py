@@ -25,6 +25,7 @@ SS_F32 = 0
 SS_BF16 = 1
 SS_MAX_WORKERS = 64
 SS_STATIC_STAGING_BYTES = 64 << 20
+SS_FLAGS_MAX_TIMEOUT_NS = 2_000_000_000
 
 SS_OK = 0
 SS_ERR_INVALID_ARG = -1
@@ -36,7 +37,8 @@ EXPORTS = ("ss_packed_words", "ss_status_string", "ss_last_cuda_error", "ss_sign
            "ss_majority_vote", "ss_signum_update", "ss_apply_vote", "ss_fused_step",
            "ss_segments_upload", "ss_fused_step_segments", "ss_apply_vote_segments",
            "ss_vote_apply", "ss_vote_apply_segments", "ss_signum_update_push", "ss_vote_tally", "ss_fused_step_host", "ss_fused_step_host_static", "ss_set_launch_option",
-           "ss_ternary_words", "ss_absmax", "ss_ternary_pack", "ss_ternary_unpack")
+           "ss_ternary_words", "ss_absmax", "ss_ternary_pack", "ss_ternary_unpack",
+           "ss_flags_signal", "ss_flags_wait", "ss_flags_signal_wait", "ss_vote_apply_guarded")
 
 
 class ss_segment(ctypes.Structure):
@@ -96,6 +98,12 @@ def lib() -> ctypes.CDLL:
     L.ss_absmax.argtypes = [vp, i32, i64, vp, vp]
     L.ss_ternary_pack.argtypes = [vp, i32, i64, vp, u64, vp, vp]
     L.ss_ternary_unpack.argtypes = [vp, i64, vp, vp, vp]
+    L.ss_flags_signal.argtypes = [vp, i32, i32, ctypes.c_uint32, vp]
+    L.ss_flags_wait.argtypes = [vp, i32, ctypes.c_uint32, u64, vp, vp]
+    L.ss_vote_apply_guarded.argtypes = [vp, i32, i64, u64, vp, f32, f32, vp, vp, vp]
+    L.ss_flags_signal_wait.argtypes = [vp, i32, i32, vp, i32, ctypes.c_uint32, u64, vp, vp]
+    for name in ("ss_flags_signal", "ss_flags_wait", "ss_flags_signal_wait", "ss_vote_apply_guarded"):
+        getattr(L, name).restype = i32
     for name in ("ss_absmax", "ss_ternary_pack", "ss_ternary_unpack"):
         getattr(L, name).restype = i32
     for name in ("ss_sign_pack", "ss_majority_vote", "ss_signum_update", "ss_apply_vote",
@@ -408,3 +416,46 @@ def ss_ternary_unpack(codes: torch.Tensor, scale_dev: torch.Tensor, out: torch.T
     _check(lib().ss_ternary_unpack(_dev(codes, torch.int32, "codes", ss_ternary_words(d)), d,
                                    _dev(scale_dev, torch.float32, "scale_dev", 1),
                                    _dev(out, torch.float32, "out"), _stream(stream)), "ss_ternary_unpack")
+
+
+# ---- flag-ordered exchange (one worker per GPU) -------------------------------------------------
+
+def flag_array(device) -> torch.Tensor:
+    """Storage for one worker's flag array: SS_MAX_WORKERS words, zeroed (epoch 0 = nothing arrived)."""
+    return torch.zeros(SS_MAX_WORKERS, dtype=torch.int32, device=device)
+
+
+def ss_flags_signal(flags: Sequence, index: int, epoch: int, stream=None) -> None:
+    """``flags`` may be tensors on this GPU or raw integer addresses of peers' flag arrays."""
+    ptrs = [p if isinstance(p, int) else _dev(p, torch.int32, "flags[%d]" % i) for i, p in enumerate(flags)]
+    _check(lib().ss_flags_signal(_ptr_array(ptrs), len(ptrs), int(index), int(epoch) & 0xFFFFFFFF,
+                                 _stream(stream)), "ss_flags_signal")
+
+
+def ss_flags_wait(flags_local: torch.Tensor, M: int, epoch: int, timeout_ns: int, status_dev: torch.Tensor,
+                  stream=None) -> None:
+    _check(lib().ss_flags_wait(_dev(flags_local, torch.int32, "flags_local"), int(M), int(epoch) & 0xFFFFFFFF,
+                               int(timeout_ns), _dev(status_dev, torch.int32, "status_dev", 1),
+                               _stream(stream)), "ss_flags_wait")
+
+
+def ss_flags_signal_wait(flags: Sequence, index: int, flags_local: torch.Tensor, M: int, epoch: int,
+                         timeout_ns: int, status_dev: torch.Tensor, stream=None) -> None:
+    ptrs = [p if isinstance(p, int) else _dev(p, torch.int32, "flags[%d]" % i) for i, p in enumerate(flags)]
+    _check(lib().ss_flags_signal_wait(_ptr_array(ptrs), len(ptrs), int(index),
+                                      _dev(flags_local, torch.int32, "flags_local"), int(M),
+                                      int(epoch) & 0xFFFFFFFF, int(timeout_ns),
+                                      _dev(status_dev, torch.int32, "status_dev", 1), _stream(stream)),
+           "ss_flags_signal_wait")
+
+
+def ss_vote_apply_guarded(packed: Sequence[torch.Tensor], param: torch.Tensor, lr: float,
+                          weight_decay: float, flip_mask: int, vote_words_out: Optional[torch.Tensor],
+                          skip_if_nonzero_dev: torch.Tensor, stream=None) -> None:
+    d = param.numel()
+    ptrs = [_words(p, d, "packed[%d]" % m) for m, p in enumerate(packed)]
+    w_ptr = None if vote_words_out is None else _words(vote_words_out, d, "vote_words_out")
+    _check(lib().ss_vote_apply_guarded(_ptr_array(ptrs), len(ptrs), d, int(flip_mask),
+                                       _dev(param, torch.float32, "param"), float(lr), float(weight_decay),
+                                       w_ptr, _dev(skip_if_nonzero_dev, torch.int32, "skip_if_nonzero_dev", 1),
+                                       _stream(stream)), "ss_vote_apply_guarded")

@@ -21,8 +21,8 @@ CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libsignsgd.so")
 OBJ_DIR = os.path.join(ROOT, "_build", "signsgd")
 
-SOURCES = ["abi.cu", "step_f32.cu", "step_bf16.cu", "vote_apply.cu", "noalloc.cu", "ternary.cu"]
-HEADERS = ["bitslice.cuh", "common.cuh", "step_kernel.cuh", "step_oct_kernel.cuh", os.path.join("..", "..", "include", "signsgd.h")]
+SOURCES = ["abi.cu", "step_f32.cu", "step_bf16.cu", "vote_apply.cu", "noalloc.cu", "ternary.cu", "exchange_flags.cu"]
+HEADERS = ["bitslice.cuh", "common.cuh", "step_kernel.cuh", "step_oct_kernel.cuh", "exchange.cuh", os.path.join("..", "..", "include", "signsgd.h")]
 
 # -fmad=false: no multiply-add contraction anywhere (the arithmetic also uses explicitly
 # rounded intrinsics); no -use_fast_math, denormals kept.

@@ -4,6 +4,7 @@
 #include <cstring>
 
 #include "common.cuh"
+#include "exchange.cuh"
 
 namespace ss {
 
@@ -280,7 +281,8 @@ int ss_apply_vote(float* param, const uint32_t* vote_words, int64_t d, float lr,
 
 static int vote_apply_common(const uint32_t* const* packed, int M, int64_t d, uint64_t flip_mask,
                              float* param, float lr, float weight_decay, const ss_segment* seg,
-                             int n_seg, uint32_t* vote_words_out, void* cuda_stream) {
+                             int n_seg, uint32_t* vote_words_out, void* cuda_stream,
+                             const uint32_t* guard = nullptr) {
     if (packed == nullptr || M < 1 || M > SS_MAX_WORKERS || !d_ok(d)) return SS_ERR_INVALID_ARG;
     if (!flip_ok(flip_mask, M)) return SS_ERR_INVALID_ARG;
     if (d == 0) return SS_OK;
@@ -298,9 +300,18 @@ static int vote_apply_common(const uint32_t* const* packed, int M, int64_t d, ui
         if (vote_words_out != nullptr && overlap(packed[m], wbytes, vote_words_out, wbytes))
             return SS_ERR_INVALID_ARG;
     }
-    return cuda_status(launch_vote_apply(packed, M, d, flip_mask, param, lr, weight_decay,
-                                         aligned(param, 16), seg, n_seg, vote_words_out,
-                                         static_cast<cudaStream_t>(cuda_stream)));
+    return cuda_status(launch_vote_apply_guarded(packed, M, d, flip_mask, param, lr, weight_decay,
+                                                 aligned(param, 16), seg, n_seg, vote_words_out, guard,
+                                                 static_cast<cudaStream_t>(cuda_stream)));
+}
+
+int ss_vote_apply_guarded(const uint32_t* const* packed, int M, int64_t d, uint64_t flip_mask,
+                          float* param, float lr, float weight_decay, uint32_t* vote_words_out,
+                          const uint32_t* skip_if_nonzero_dev, void* cuda_stream) {
+    if (skip_if_nonzero_dev == nullptr) return SS_ERR_INVALID_ARG;
+    if (!aligned(skip_if_nonzero_dev, 4)) return SS_ERR_MISALIGNED;
+    return vote_apply_common(packed, M, d, flip_mask, param, lr, weight_decay, nullptr, 0,
+                             vote_words_out, cuda_stream, skip_if_nonzero_dev);
 }
 
 int ss_vote_apply(const uint32_t* const* packed, int M, int64_t d, uint64_t flip_mask, float* param,

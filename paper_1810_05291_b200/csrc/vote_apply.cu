@@ -9,6 +9,7 @@
 
 #include "bitslice.cuh"
 #include "common.cuh"
+#include "exchange.cuh"
 
 namespace ss {
 
@@ -189,7 +190,14 @@ struct VoteApplyArgs {
     const ss_segment* seg;
     int n_seg;
     int M;
+    const uint32_t* guard;  // may be null; a non-zero word there makes the whole launch a no-op
 };
+
+// true if the launch has been called off: the word at `guard` (written by an earlier kernel of the
+// stream, e.g. a wait for the other workers that ran out of time) is not zero
+__device__ __forceinline__ bool called_off(const uint32_t* guard) {
+    return guard != nullptr && *reinterpret_cast<const volatile uint32_t*>(guard) != 0u;
+}
 
 // Pair form (every packed pointer and the vote output 8-byte aligned, x 16-byte aligned). A warp
 // owns a tile of 64 packed words = 2048 coordinates: lane l loads words 2l and 2l+1 of every
@@ -279,6 +287,7 @@ __device__ __forceinline__ void vote_apply_pair_tile(const VoteApplyArgs<CAP>& a
 template <int CAP, bool EXACT, bool SEG>
 __global__ void __launch_bounds__(256, 4)
 vote_apply_pair_kernel(const __grid_constant__ VoteApplyArgs<CAP> a) {
+    if (called_off(a.guard)) return;
     const int M = EXACT ? CAP : a.M;
     const int lane = threadIdx.x & 31;
     const int64_t n_full = a.d >> 11;                          // tiles whose 2048 coordinates all exist
@@ -305,6 +314,7 @@ vote_apply_pair_kernel(const __grid_constant__ VoteApplyArgs<CAP> a) {
 template <bool VEC, bool SEG>
 __global__ void __launch_bounds__(256)
 vote_apply_word_kernel(const __grid_constant__ VoteApplyArgs<SS_MAX_WORKERS> a) {
+    if (called_off(a.guard)) return;
     constexpr int CAP = SS_MAX_WORKERS;
     const int M = a.M;
     const int lane = threadIdx.x & 31;
@@ -376,7 +386,8 @@ vote_apply_word_kernel(const __grid_constant__ VoteApplyArgs<SS_MAX_WORKERS> a) 
 template <int CAP>
 void fill_vote_apply_args(VoteApplyArgs<CAP>& a, const uint32_t* const* packed, int M, int64_t d,
                           uint64_t flip, float* x, float lr, float wd, const ss_segment* seg, int n_seg,
-                          uint32_t* vote) {
+                          uint32_t* vote, const uint32_t* guard) {
+    a.guard = guard;
     for (int m = 0; m < CAP; ++m) a.p[m] = m < M ? packed[m] : nullptr;
     a.out = vote;
     a.x = x;
@@ -392,9 +403,9 @@ void fill_vote_apply_args(VoteApplyArgs<CAP>& a, const uint32_t* const* packed, 
 template <int CAP, bool EXACT, bool SEG>
 cudaError_t launch_vote_apply_pair(const uint32_t* const* packed, int M, int64_t d, uint64_t flip,
                                    float* x, float lr, float wd, const ss_segment* seg, int n_seg,
-                                   uint32_t* vote, cudaStream_t st) {
+                                   uint32_t* vote, const uint32_t* guard, cudaStream_t st) {
     VoteApplyArgs<CAP> a;
-    fill_vote_apply_args(a, packed, M, d, flip, x, lr, wd, seg, n_seg, vote);
+    fill_vote_apply_args(a, packed, M, d, flip, x, lr, wd, seg, n_seg, vote, guard);
     const int threads = launch_threads();
     const int64_t tiles = (((d + 31) >> 5) + 63) >> 6;
     const int64_t per_block = threads / 32;
@@ -409,9 +420,9 @@ cudaError_t launch_vote_apply_pair(const uint32_t* const* packed, int M, int64_t
 template <bool VEC, bool SEG>
 cudaError_t launch_vote_apply_word(const uint32_t* const* packed, int M, int64_t d, uint64_t flip,
                                    float* x, float lr, float wd, const ss_segment* seg, int n_seg,
-                                   uint32_t* vote, cudaStream_t st) {
+                                   uint32_t* vote, const uint32_t* guard, cudaStream_t st) {
     VoteApplyArgs<SS_MAX_WORKERS> a;
-    fill_vote_apply_args(a, packed, M, d, flip, x, lr, wd, seg, n_seg, vote);
+    fill_vote_apply_args(a, packed, M, d, flip, x, lr, wd, seg, n_seg, vote, guard);
     const int threads = launch_threads();
     const int64_t tiles = (((d + 31) >> 5) + 31) >> 5;
     const int64_t per_block = threads / 32;
@@ -426,24 +437,30 @@ cudaError_t launch_vote_apply_word(const uint32_t* const* packed, int M, int64_t
 template <bool SEG>
 cudaError_t launch_vote_apply_seg(const uint32_t* const* packed, int M, int64_t d, uint64_t flip,
                                   float* x, float lr, float wd, bool vec, const ss_segment* seg,
-                                  int n_seg, uint32_t* vote, cudaStream_t st) {
+                                  int n_seg, uint32_t* vote, const uint32_t* guard, cudaStream_t st) {
     bool pair = vec && (vote == nullptr || (reinterpret_cast<uintptr_t>(vote) & 7) == 0);
     for (int m = 0; m < M; ++m) pair = pair && (reinterpret_cast<uintptr_t>(packed[m]) & 7) == 0;
     if (!pair)
-        return vec ? launch_vote_apply_word<true, SEG>(packed, M, d, flip, x, lr, wd, seg, n_seg, vote, st)
-                   : launch_vote_apply_word<false, SEG>(packed, M, d, flip, x, lr, wd, seg, n_seg, vote, st);
+        return vec ? launch_vote_apply_word<true, SEG>(packed, M, d, flip, x, lr, wd, seg, n_seg, vote, guard, st)
+                   : launch_vote_apply_word<false, SEG>(packed, M, d, flip, x, lr, wd, seg, n_seg, vote, guard, st);
 #define SS_VA(CAPV, EX) \
-    launch_vote_apply_pair<CAPV, EX, SEG>(packed, M, d, flip, x, lr, wd, seg, n_seg, vote, st)
+    launch_vote_apply_pair<CAPV, EX, SEG>(packed, M, d, flip, x, lr, wd, seg, n_seg, vote, guard, st)
     SS_DISPATCH_WORKERS(M, SS_VA);
 #undef SS_VA
+}
+
+cudaError_t launch_vote_apply_guarded(const uint32_t* const* packed, int M, int64_t d, uint64_t flip,
+                                      float* x, float lr, float wd, bool vec, const ss_segment* seg,
+                                      int n_seg, uint32_t* vote, const uint32_t* guard, cudaStream_t st) {
+    return seg != nullptr
+               ? launch_vote_apply_seg<true>(packed, M, d, flip, x, lr, wd, vec, seg, n_seg, vote, guard, st)
+               : launch_vote_apply_seg<false>(packed, M, d, flip, x, lr, wd, vec, seg, n_seg, vote, guard, st);
 }
 
 cudaError_t launch_vote_apply(const uint32_t* const* packed, int M, int64_t d, uint64_t flip,
                               float* x, float lr, float wd, bool vec, const ss_segment* seg,
                               int n_seg, uint32_t* vote, cudaStream_t st) {
-    return seg != nullptr
-               ? launch_vote_apply_seg<true>(packed, M, d, flip, x, lr, wd, vec, seg, n_seg, vote, st)
-               : launch_vote_apply_seg<false>(packed, M, d, flip, x, lr, wd, vec, seg, n_seg, vote, st);
+    return launch_vote_apply_guarded(packed, M, d, flip, x, lr, wd, vec, seg, n_seg, vote, nullptr, st);
 }
 
 // ---- the tally itself: V = sum_m sign(v_m) per coordinate as int8 (a diagnostic: the margin by

@@ -143,6 +143,8 @@ class MajorityVoteWorker:
         self.vote = torch.zeros(self.ex.W, dtype=torch.int32, device=param.device)
         self.push_dests = None
         self.barrier = None
+        self.flags = None            # flag-ordered push: see set_flag_exchange
+        self.epoch = 0
         self.on_phase = on_phase
         if mode == "push" and beta is None:
             raise ValueError("push mode carries the momentum kernel: use it with Signum (beta set)")
@@ -162,7 +164,38 @@ class MajorityVoteWorker:
         self.push_dests = list(dests)
         self.barrier = barrier
 
-    def connect_push(self, group=None, barrier: str = "collective") -> None:
+    def set_flag_exchange(self, recv_bufs, dests, flag_dests, flags_local, timeout_ns: int = 1_000_000_000,
+                          signal_with_wait: bool = False) -> None:
+        """push mode without any collective: the flag-ordered exchange of ``ss_flags_signal`` /
+        ``ss_flags_wait``. ``recv_bufs`` are this worker's two receive buffers (used alternately by
+        the parity of the step, world * W_pad words each); ``dests[parity][m]`` is the address
+        (tensor or int) of this worker's slot in worker m's buffer of that parity;
+        ``flag_dests[m]`` is worker m's flag array and ``flags_local`` this worker's own. After a
+        step whose wait ran out of time the update is skipped as a whole; ``check()`` tells.
+        ``signal_with_wait``: raise the flag in the launch that waits (``ss_flags_signal_wait``, one
+        launch fewer per step) instead of right after the push; only for workers whose ``finish``
+        follows their own ``pack_local`` without waiting for other workers' calls on this host."""
+        world = self.ex.world
+        if len(recv_bufs) != 2 or len(dests) != 2 or any(len(x) != world for x in dests) or len(flag_dests) != world:
+            raise ValueError("need two receive buffers, two lists of one destination per worker, one flag array per worker")
+        self.flags = dict(recv=list(recv_bufs), dests=[list(dests[0]), list(dests[1])], flag_dests=list(flag_dests),
+                          local=flags_local, timeout_ns=int(timeout_ns), fused=bool(signal_with_wait),
+                          status=torch.zeros(1, dtype=torch.int32, device=self.x.device))
+
+    def check(self) -> None:
+        """Flag-ordered push: waits for the stream and raises if the last wait ran out of time
+        (RuntimeError naming the lowest worker whose packed signs had not arrived)."""
+        if self.flags is None:
+            return
+        if self.x.is_cuda:
+            torch.cuda.synchronize(self.x.device)
+        status = int(self.flags["status"].item())
+        if status != 0:
+            raise RuntimeError("majority vote step %d: the packed signs of worker %d did not arrive within "
+                               "%.3f s; the parameter update of that step was skipped"
+                               % (self.epoch, status - 1, self.flags["timeout_ns"] * 1e-9))
+
+    def connect_push(self, group=None, barrier: str = "collective", timeout_ns: int = 1_000_000_000) -> None:
         """push mode across GPUs: allocates the receive buffer in symmetric memory
         (``torch.distributed._symmetric_memory``), exchanges its addresses over ``group``, and
         points this worker's push at its own slot in every peer's buffer. Every worker of the
@@ -174,14 +207,36 @@ class MajorityVoteWorker:
         has reached it, and a worker that never arrives ends it with the process group's timeout
         error on the host. ``barrier="signal"``: the symmetric-memory handle's own barrier, a
         spin on a flag in the peers' signal pads inside a kernel, with the library's own timeout;
-        lower latency, kept as an explicit choice."""
+        lower latency, kept as an explicit choice. ``barrier="flags"``: no barrier and no collective
+        at all: two receive buffers used alternately and one flag per worker, raised by
+        ``ss_flags_signal`` after the push and awaited, for at most ``timeout_ns``, by
+        ``ss_flags_wait`` before the vote (see ``set_flag_exchange``)."""
         import torch.distributed._symmetric_memory as symm
         if self.ex.mode != "push":
             raise RuntimeError("connect_push is for push mode")
-        if barrier not in ("collective", "signal"):
-            raise ValueError("barrier must be 'collective' or 'signal'")
+        if barrier not in ("collective", "signal", "flags"):
+            raise ValueError("barrier must be 'collective', 'signal' or 'flags'")
         group = group if group is not None else dist.group.WORLD
         ex = self.ex
+        if barrier == "flags":
+            n_buf = ex.world * ex.W_pad
+            n_flags = self.B.SS_MAX_WORKERS
+            buf = symm.empty(2 * n_buf + n_flags, dtype=torch.int32, device=self.x.device)
+            buf.zero_()
+            handle = symm.rendezvous(buf, group)
+            self._symmetric = (buf, handle)
+            base = [int(handle.buffer_ptrs[m]) for m in range(ex.world)]
+            slot = ex.rank * ex.W_pad * 4
+            dests = [[base[m] + parity * n_buf * 4 + slot for m in range(ex.world)] for parity in (0, 1)]
+            flag_dests = [base[m] + 2 * n_buf * 4 for m in range(ex.world)]
+            # every worker's buffers and flags are zero before anyone pushes: a host-side barrier,
+            # once, at set-up
+            if self.x.is_cuda:
+                torch.cuda.synchronize(self.x.device)
+            dist.barrier(group)
+            self.set_flag_exchange([buf[:n_buf], buf[n_buf:2 * n_buf]], dests, flag_dests,
+                                   buf[2 * n_buf: 2 * n_buf + n_flags], timeout_ns, signal_with_wait=True)
+            return
         buf = symm.empty(ex.world * ex.W_pad, dtype=torch.int32, device=self.x.device)
         buf.zero_()
         handle = symm.rendezvous(buf, group)
@@ -196,9 +251,18 @@ class MajorityVoteWorker:
 
     def pack_local(self, grad: torch.Tensor, stream=None) -> None:
         """Worker side: v <- (1 - beta) g + beta v, sign(v) packed into the send buffer."""
+        if self.ex.mode == "push" and self.flags is not None:
+            self.epoch += 1
+            fl = self.flags
+            self.B.ss_signum_update_push(grad, self.momentum, self.beta, fl["dests"][self.epoch & 1], stream)
+            self._phase("kernel:pack")
+            if not fl["fused"]:
+                self.B.ss_flags_signal(fl["flag_dests"], self.ex.rank, self.epoch, stream)
+                self._phase("exchange:signal")
+            return
         if self.ex.mode == "push":
             if self.push_dests is None:
-                raise RuntimeError("push mode: call set_push_destinations first")
+                raise RuntimeError("push mode: call set_push_destinations, set_flag_exchange or connect_push first")
             self.B.ss_signum_update_push(grad, self.momentum, self.beta, self.push_dests, stream)
         elif self.momentum is not None:
             self.B.ss_signum_update(grad, self.momentum, self.beta, self.ex.local_words(), stream)
@@ -223,6 +287,19 @@ class MajorityVoteWorker:
         """Receive what the update needs (all packed vectors, or the voted slices), update the
         parameters, and return the packed vote of the whole vector."""
         B, ex = self.B, self.ex
+        if ex.mode == "push" and self.flags is not None:
+            fl = self.flags
+            ex.gathered = fl["recv"][self.epoch & 1]
+            if fl["fused"]:
+                B.ss_flags_signal_wait(fl["flag_dests"], ex.rank, fl["local"], ex.world, self.epoch,
+                                       fl["timeout_ns"], fl["status"], stream)
+            else:
+                B.ss_flags_wait(fl["local"], ex.world, self.epoch, fl["timeout_ns"], fl["status"], stream)
+            self._phase("exchange:wait")
+            B.ss_vote_apply_guarded(ex.worker_rows(), self.x, self.lr, self.weight_decay, flip_mask,
+                                    self.vote, fl["status"], stream)
+            self._phase("kernel:vote_apply")
+            return self.vote
         if ex.mode == "push":
             self.barrier()
             self._phase("exchange:barrier")

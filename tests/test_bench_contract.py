@@ -114,16 +114,21 @@ def test_traffic_is_null_once_the_kernel_sources_have_changed(monkeypatch):
 
 
 @pytest.mark.gpu
-@pytest.mark.parametrize("layout", ["allgather", "sharded", "push"])
+@pytest.mark.parametrize("layout", ["allgather", "sharded", "push", "push:flags"])
 def test_worker_per_gpu_mode_runs_on_one_rank(layout):
-    r = _run(["--mode", "worker-per-gpu", "--layout", layout, "--steps", "4", "--warmup", "3", "--d", "1000008"])
+    extra = []
+    if ":" in layout:
+        layout, barrier = layout.split(":")
+        extra = ["--push-barrier", barrier]
+    r = _run(["--mode", "worker-per-gpu", "--layout", layout, "--steps", "4", "--warmup", "3", "--d", "1000008"] + extra)
     assert r["mode"] == "worker-per-gpu" and r["layout"] == layout and r["n_gpus"] == 1
     assert r["config"]["M"] == 1 and r["value"] > 0 and r["ms_per_step"] > 0
     assert r["kernel_ms_per_step"] > 0 and r["exchange_ms_per_step"] >= 0
     assert r["kernel_ms_per_step"] + r["exchange_ms_per_step"] <= r["ms_per_step"] * 1.05
     assert r["bytes_received_per_worker_per_step"] == 0          # a lone worker receives nothing
     assert r["paper_bits_per_iteration_whole_system"] == 2 * 1000008
-    assert r["gpu_launches"] == {"allgather": 2, "sharded": 3, "push": 2}[layout] * 4
+    per_step = 3 if extra else {"allgather": 2, "sharded": 3, "push": 2}[layout]
+    assert r["gpu_launches"] == per_step * 4
 
 
 @pytest.mark.gpu

@@ -8,6 +8,7 @@ M-worker step gives, in both exchange layouts.
 """
 import os
 import socket
+import time
 
 import numpy as np
 import pytest
@@ -134,11 +135,49 @@ class OracleKernels:
             self._u32(vote_words_out)[:] = vote
 
 
+    # ---- flag-ordered exchange: the flags are words of shared memory that other processes write
+    SS_MAX_WORKERS = 64
+
+    def ss_flags_signal(self, flags, index, epoch, stream=None):
+        self.calls.append("ss_flags_signal")
+        for f in flags:
+            f[index] = epoch
+
+    def ss_flags_wait(self, flags_local, M, epoch, timeout_ns, status_dev, stream=None):
+        self.calls.append("ss_flags_wait")
+        deadline = time.monotonic() + timeout_ns * 1e-9
+        while True:
+            seen = flags_local[:M].clone()
+            late = (seen < epoch).nonzero()
+            if late.numel() == 0:
+                status_dev[0] = 0
+                return
+            if time.monotonic() > deadline:
+                status_dev[0] = int(late[0]) + 1
+                return
+            time.sleep(0.001)
+
+    def ss_flags_signal_wait(self, flags, index, flags_local, M, epoch, timeout_ns, status_dev, stream=None):
+        self.ss_flags_signal(flags, index, epoch)
+        self.ss_flags_wait(flags_local, M, epoch, timeout_ns, status_dev)
+
+    def ss_vote_apply_guarded(self, packed, param, lr, weight_decay, flip_mask, vote_words_out,
+                              skip_if_nonzero_dev, stream=None):
+        self.calls.append("ss_vote_apply_guarded")
+        if int(skip_if_nonzero_dev[0]) != 0:
+            return
+        self.calls.pop()
+        self.ss_vote_apply(packed, param, lr, weight_decay, flip_mask, vote_words_out, stream)
+        self.calls[-1] = "ss_vote_apply_guarded"
+
+
 EXPECTED_ORDER = {
     "allgather": ["start", "kernel:pack", "exchange:all_gather", "kernel:vote_apply"],
     "sharded": ["start", "kernel:pack", "exchange:all_to_all", "kernel:vote", "exchange:all_gather",
                 "kernel:apply"],
     "push": ["start", "kernel:pack", "exchange:barrier", "kernel:vote_apply", "exchange:barrier"],
+    "push-flags": ["start", "kernel:pack", "exchange:signal", "exchange:wait", "kernel:vote_apply"],
+    "push-flags-fused": ["start", "kernel:pack", "exchange:wait", "kernel:vote_apply"],
 }
 
 
@@ -153,9 +192,18 @@ def _worker_main(rank, world, port, d, mode, flip, beta, shared):
         x0 = rng.standard_normal(d).astype(np.float32)
         phases = []
         kernels = OracleKernels()
-        w = MajorityVoteWorker(torch.from_numpy(x0.copy()), beta, lr, wd, mode, world=world, rank=rank,
-                               kernels=kernels, on_phase=phases.append)
-        if mode == "push":
+        w = MajorityVoteWorker(torch.from_numpy(x0.copy()), beta, lr, wd, mode.split("-")[0], world=world,
+                               rank=rank, kernels=kernels, on_phase=phases.append)
+        if mode.startswith("push-flags"):
+            # two receive buffers and one flag array per rank, all in shared memory; no barrier, no
+            # collective: the ranks are ordered by the flags alone
+            n = world * w.ex.W_pad
+            slot = lambda buf: buf[rank * w.ex.W_pad: rank * w.ex.W_pad + w.ex.W]
+            w.set_flag_exchange([shared[rank][0], shared[rank][1]],
+                                [[slot(shared[m][parity]) for m in range(world)] for parity in (0, 1)],
+                                [shared[m][2] for m in range(world)], shared[rank][2], timeout_ns=20_000_000_000,
+                                signal_with_wait=mode.endswith("fused"))
+        elif mode == "push":
             # the receive buffers live in shared memory: a stand-in for peer-mapped device memory,
             # written by the other ranks' processes and ordered only by the barrier
             w.ex.gathered = shared[rank]
@@ -168,7 +216,10 @@ def _worker_main(rank, world, port, d, mode, flip, beta, shared):
             grads = [rng.standard_normal(d).astype(np.float32) for _ in range(world)]
             want = oracle.fused_step(grads, ref_v, ref_x, beta if beta is not None else 0.0, lr, wd, flip)
             del phases[:]
+            if mode.startswith("push-flags") and rank == 1:
+                time.sleep(0.05 * step)              # a straggler: the others must wait for its flag
             vote = w.step(torch.from_numpy(grads[rank].copy()), flip)
+            w.check()
             assert phases == EXPECTED_ORDER[mode], phases
             assert np.array_equal(_as_u32(vote), want), "rank %d step %d: vote differs" % (rank, step)
             assert np.array_equal(w.x.numpy().view(np.uint32), ref_x.view(np.uint32)), "rank %d: x differs" % rank
@@ -177,7 +228,9 @@ def _worker_main(rank, world, port, d, mode, flip, beta, shared):
         want_calls = {"allgather": ["ss_signum_update" if beta is not None else "ss_sign_pack", "ss_vote_apply"],
                       "sharded": ["ss_signum_update" if beta is not None else "ss_sign_pack",
                                   "ss_majority_vote", "ss_apply_vote"],
-                      "push": ["ss_signum_update_push", "ss_vote_apply"]}[mode]
+                      "push": ["ss_signum_update_push", "ss_vote_apply"],
+                      "push-flags": ["ss_signum_update_push", "ss_flags_signal", "ss_flags_wait",
+                                     "ss_vote_apply_guarded"]}[mode.replace("-fused", "")]
         if mode == "sharded" and w.ex.slice_coordinates() == 0:
             want_calls = [c for c in want_calls if c != "ss_majority_vote"]
         assert kernels.calls == want_calls * 3, kernels.calls
@@ -188,13 +241,68 @@ def _worker_main(rank, world, port, d, mode, flip, beta, shared):
 @pytest.mark.parametrize("mode,world,d,flip,beta", [
     ("allgather", 2, 100_003, 0b01, 0.9), ("allgather", 3, 70, 0, None),
     ("sharded", 2, 1000, 0, 0.9), ("sharded", 3, 33, 0b010, None), ("sharded", 3, 100_003, 0b100, 0.9),
-    ("push", 2, 100_003, 0b10, 0.9), ("push", 3, 1000, 0, 0.9)])
+    ("push", 2, 100_003, 0b10, 0.9), ("push", 3, 1000, 0, 0.9),
+    ("push-flags", 2, 100_003, 0b10, 0.9), ("push-flags", 3, 1000, 0, 0.9),
+    ("push-flags-fused", 3, 100_003, 0b001, 0.9)])
 def test_majority_vote_worker_step_over_gloo(mode, world, d, flip, beta):
     shared = None
+    W_pad = PackedExchange(d, world, 0, "meta", "push").W_pad
     if mode == "push":
-        W_pad = PackedExchange(d, world, 0, "meta", "push").W_pad
         shared = [torch.zeros(world * W_pad, dtype=torch.int32).share_memory_() for _ in range(world)]
+    if mode.startswith("push-flags"):
+        shared = [[torch.zeros(world * W_pad, dtype=torch.int32).share_memory_(),
+                   torch.zeros(world * W_pad, dtype=torch.int32).share_memory_(),
+                   torch.zeros(64, dtype=torch.int32).share_memory_()] for _ in range(world)]
     mp.spawn(_worker_main, args=(world, _free_port(), d, mode, flip, beta, shared), nprocs=world, join=True)
+
+
+def _leaver_main(rank, world, port, d, shared, out_dir):
+    """Failure made on the host: rank 1 takes part in step 1 and then leaves (between steps, with
+    nothing of its own in flight). Rank 0's wait of step 2 must run out of time, name worker 1, and
+    leave the parameters of step 1 untouched."""
+    os.environ["MASTER_ADDR"] = "127.0.0.1"
+    os.environ["MASTER_PORT"] = str(port)
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    try:
+        rng = np.random.default_rng(99)
+        x0 = rng.standard_normal(d).astype(np.float32)
+        w = MajorityVoteWorker(torch.from_numpy(x0.copy()), 0.9, 1e-3, 0.0, "push", world=world, rank=rank,
+                               kernels=OracleKernels())
+        slot = lambda buf: buf[rank * w.ex.W_pad: rank * w.ex.W_pad + w.ex.W]
+        w.set_flag_exchange([shared[rank][0], shared[rank][1]],
+                            [[slot(shared[m][parity]) for m in range(world)] for parity in (0, 1)],
+                            [shared[m][2] for m in range(world)], shared[rank][2], timeout_ns=300_000_000)
+        grads = [rng.standard_normal(d).astype(np.float32) for _ in range(world)]
+        w.step(torch.from_numpy(grads[rank].copy()))
+        w.check()
+        if rank == 1:
+            return                                    # leaves; never pushes again
+        x_after_step_1 = w.x.clone()
+        t0 = time.monotonic()
+        w.step(torch.from_numpy(grads[rank].copy()))
+        waited = time.monotonic() - t0
+        try:
+            w.check()
+            outcome = "no error"
+        except RuntimeError as e:
+            outcome = str(e)
+        with open(os.path.join(out_dir, "outcome.txt"), "w") as f:
+            f.write("%s\n%.3f\n%d\n" % (outcome, waited, int(torch.equal(w.x, x_after_step_1))))
+    finally:
+        dist.destroy_process_group()
+
+
+def test_a_worker_that_leaves_is_detected_by_the_bounded_wait(tmp_path):
+    d, world = 1000, 2
+    W_pad = PackedExchange(d, world, 0, "meta", "push").W_pad
+    shared = [[torch.zeros(world * W_pad, dtype=torch.int32).share_memory_(),
+               torch.zeros(world * W_pad, dtype=torch.int32).share_memory_(),
+               torch.zeros(64, dtype=torch.int32).share_memory_()] for _ in range(world)]
+    mp.spawn(_leaver_main, args=(world, _free_port(), d, shared, str(tmp_path)), nprocs=world, join=True)
+    outcome, waited, unchanged = open(tmp_path / "outcome.txt").read().strip().split("\n")
+    assert "worker 1 did not arrive" in outcome and "step 2" in outcome
+    assert 0.25 < float(waited) < 5.0                # waited about the time limit, then gave up
+    assert unchanged == "1"                          # the update of the failed step was skipped as a whole
 
 
 @pytest.mark.parametrize("d,world", [(1, 1), (1, 4), (31, 2), (32, 2), (33, 2), (1000, 3), (1024, 4),

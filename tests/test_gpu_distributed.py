@@ -130,7 +130,7 @@ def test_one_rank_nccl_group_runs_the_real_collectives(mode):
         dist.destroy_process_group()
 
 
-@pytest.mark.parametrize("barrier", ["collective", "signal"])
+@pytest.mark.parametrize("barrier", ["collective", "signal", "flags"])
 def test_push_mode_over_symmetric_memory_with_one_rank(barrier):
     """The symmetric-memory wiring of push mode on a one-rank group: the receive buffer is a
     symmetric allocation, the push goes to the address the rendezvous reports, and the barrier (a
@@ -158,10 +158,130 @@ def test_push_mode_over_symmetric_memory_with_one_rank(barrier):
             want = oracle.fused_step([g], ref_v, ref_x, 0.9, 1e-3)
             vote = w.step(torch.from_numpy(g).to(DEV))
             torch.cuda.synchronize()
+            w.check()
             assert np.array_equal(vote.cpu().numpy().view(np.uint32), want)
             assert np.array_equal(w.x.cpu().numpy().view(np.uint32), ref_x.view(np.uint32))
     finally:
         dist.destroy_process_group()
+
+
+def _flag_workers(M, d, x0, timeout_ns):
+    """M workers in one process wired for the flag-ordered push: two receive buffers and a flag
+    array each, every destination a local tensor."""
+    from paper_1810_05291_b200 import binding as B
+    workers = [MajorityVoteWorker(torch.from_numpy(x0.copy()).to(DEV), 0.9, 1e-3, 0.0, "push", world=M, rank=m)
+               for m in range(M)]
+    n = workers[0].ex.world * workers[0].ex.W_pad
+    bufs = [[torch.zeros(n, dtype=torch.int32, device=DEV) for _ in (0, 1)] for _ in range(M)]
+    flags = [B.flag_array(DEV) for _ in range(M)]
+    for m, w in enumerate(workers):
+        slot = lambda buf: buf[m * w.ex.W_pad: m * w.ex.W_pad + w.ex.W]
+        w.set_flag_exchange(bufs[m], [[slot(bufs[p][parity]) for p in range(M)] for parity in (0, 1)],
+                            flags, flags[m], timeout_ns)
+    return workers
+
+
+@pytest.mark.parametrize("M,d,flip", [(3, 1000, 0), (7, 100_003, 0b0100000), (15, 32 * 3000 + 8, 0)])
+def test_flag_ordered_push_in_one_process(M, d, flip):
+    """Push, signal, bounded wait, guarded vote + update, with no barrier and no collective. On one
+    GPU the workers' kernels run one after another on one stream, so every wait finds its flags
+    already raised: this checks the flags, epochs, alternating buffers and the guard, not concurrency."""
+    rng = np.random.default_rng(11 * M + d)
+    x0 = rng.standard_normal(d).astype(np.float32)
+    workers = _flag_workers(M, d, x0, timeout_ns=200_000_000)
+    ref_x = x0.copy()
+    ref_v = [np.zeros(d, dtype=np.float32) for _ in range(M)]
+    for step in range(5):                                  # both buffer parities, several epochs
+        grads = [rng.standard_normal(d).astype(np.float32) for _ in range(M)]
+        want = oracle.fused_step(grads, ref_v, ref_x, 0.9, 1e-3, 0.0, flip)
+        for m, w in enumerate(workers):
+            w.pack_local(torch.from_numpy(grads[m]).to(DEV))
+        votes = [w.finish(flip) for w in workers]
+        for m, w in enumerate(workers):
+            w.check()
+            assert np.array_equal(votes[m].cpu().numpy().view(np.uint32), want)
+            assert np.array_equal(w.x.cpu().numpy().view(np.uint32), ref_x.view(np.uint32))
+            assert np.array_equal(w.momentum.cpu().numpy().view(np.uint32), ref_v[m].view(np.uint32))
+            assert w.flags["local"][:M].tolist() == [step + 1] * M
+
+
+def test_wait_runs_out_when_a_worker_never_signals():
+    """The failure is made on the host: worker 2 simply does not take part in the step. Worker 0's
+    wait must come back after its time limit, name worker 2, leave x and the vote buffer as they
+    were, and leave the GPU usable."""
+    import time
+
+    from paper_1810_05291_b200 import binding as B
+    M, d = 3, 50_000
+    rng = np.random.default_rng(5)
+    x0 = rng.standard_normal(d).astype(np.float32)
+    workers = _flag_workers(M, d, x0, timeout_ns=30_000_000)          # 30 ms
+    grads = [rng.standard_normal(d).astype(np.float32) for _ in range(M)]
+    for m in (0, 1):
+        workers[m].pack_local(torch.from_numpy(grads[m]).to(DEV))
+    w = workers[0]
+    w.vote.fill_(-1)
+    torch.cuda.synchronize()
+    t0 = time.monotonic()
+    w.finish(0)
+    torch.cuda.synchronize()
+    waited = time.monotonic() - t0
+    assert 0.025 < waited < 2.0
+    assert int(w.flags["status"].item()) == 3                           # 1 + the missing worker
+    with pytest.raises(RuntimeError, match="worker 2 did not arrive"):
+        w.check()
+    assert np.array_equal(w.x.cpu().numpy().view(np.uint32), x0.view(np.uint32))   # nothing was updated
+    assert bool((w.vote == -1).all())
+    # the context is intact: an ordinary call still runs and is right
+    g = torch.from_numpy(grads[0]).to(DEV)
+    words = torch.zeros(B.ss_packed_words(d), dtype=torch.int32, device=DEV)
+    B.ss_sign_pack(g, words)
+    assert np.array_equal(words.cpu().numpy().view(np.uint32), oracle.sign_pack(grads[0]))
+    # the late worker arrives: the same epoch's wait now succeeds and the step goes through
+    workers[2].pack_local(torch.from_numpy(grads[2]).to(DEV))
+    w.finish(0)
+    w.check()
+    ref_x, ref_v = x0.copy(), [np.zeros(d, dtype=np.float32) for _ in range(M)]
+    want = oracle.fused_step(grads, ref_v, ref_x, 0.9, 1e-3)
+    assert np.array_equal(w.vote.cpu().numpy().view(np.uint32), want)
+    assert np.array_equal(w.x.cpu().numpy().view(np.uint32), ref_x.view(np.uint32))
+
+
+def test_flag_epochs_compare_as_serial_numbers():
+    from paper_1810_05291_b200 import binding as B
+    flags = B.flag_array(DEV)
+    status = torch.full((1,), 77, dtype=torch.int32, device=DEV)
+    flags[0], flags[1] = 5, 5
+    B.ss_flags_wait(flags, 2, 0xFFFFFFFE, 1_000_000, status)          # 5 is "after" 2^32 - 2
+    assert int(status.item()) == 0
+    flags[1] = -1                                                      # 2^32 - 1 is "before" 2
+    B.ss_flags_wait(flags, 2, 2, 1_000_000, status)
+    assert int(status.item()) == 2
+    B.ss_flags_signal([flags], 1, 3)
+    B.ss_flags_wait(flags, 2, 3, 1_000_000, status)
+    assert int(status.item()) == 0 and flags[:3].tolist() == [5, 3, 0]
+
+
+def test_guarded_vote_apply_skips_everything_or_nothing():
+    from paper_1810_05291_b200 import binding as B
+    M, d = 7, 64 * 32 * 3 + 45
+    gen = torch.Generator(device=DEV).manual_seed(8)
+    W = B.ss_packed_words(d)
+    packed = [torch.randint(-(1 << 31), 1 << 31, (W,), generator=gen, device=DEV, dtype=torch.int64).to(torch.int32)
+              for _ in range(M)]
+    x0 = torch.randn(d, generator=gen, device=DEV)
+    for misalign in (0, 1):                                            # pair kernel and word kernel
+        xs = torch.zeros(d + misalign, device=DEV)[misalign:]
+        xs.copy_(x0)
+        vote = torch.full((W,), -1, dtype=torch.int32, device=DEV)
+        guard = torch.full((1,), 4, dtype=torch.int32, device=DEV)
+        B.ss_vote_apply_guarded(packed, xs, 1e-3, 0.0, 0b11, vote, guard)
+        assert torch.equal(xs, x0) and bool((vote == -1).all())
+        guard.zero_()
+        B.ss_vote_apply_guarded(packed, xs, 1e-3, 0.0, 0b11, vote, guard)
+        xr, vr = x0.clone(), torch.zeros(W, dtype=torch.int32, device=DEV)
+        B.ss_vote_apply(packed, xr, 1e-3, 0.0, 0b11, vr)
+        assert torch.equal(xs, xr) and torch.equal(vote, vr)
 
 
 def _nccl_worker(rank, world, port, mode, d, beta, flip, errors):
@@ -176,9 +296,9 @@ def _nccl_worker(rank, world, port, mode, d, beta, flip, errors):
         try:
             rng = np.random.default_rng(5000 + d + world)
             x0 = rng.standard_normal(d).astype(np.float32)
-            w = MajorityVoteWorker(torch.from_numpy(x0.copy()).to(dev), beta, 1e-3, 0.01, mode)
-            if mode == "push":
-                w.connect_push()
+            w = MajorityVoteWorker(torch.from_numpy(x0.copy()).to(dev), beta, 1e-3, 0.01, mode.split("-")[0])
+            if mode.startswith("push"):
+                w.connect_push(barrier="flags" if mode == "push-flags" else "collective")
             ref_x = x0.copy()
             ref_v = [np.zeros(d, dtype=np.float32) for _ in range(world)] if beta is not None else None
             for step in range(4):
@@ -186,6 +306,7 @@ def _nccl_worker(rank, world, port, mode, d, beta, flip, errors):
                 want = oracle.fused_step(grads, ref_v, ref_x, beta if beta is not None else 0.0, 1e-3, 0.01, flip)
                 vote = w.step(torch.from_numpy(grads[rank]).to(dev), flip)
                 torch.cuda.synchronize()
+                w.check()
                 assert np.array_equal(vote.cpu().numpy().view(np.uint32), want), "vote, step %d" % step
                 assert np.array_equal(w.x.cpu().numpy().view(np.uint32), ref_x.view(np.uint32)), "x, step %d" % step
                 if beta is not None:
@@ -198,7 +319,8 @@ def _nccl_worker(rank, world, port, mode, d, beta, flip, errors):
 
 
 @pytest.mark.parametrize("world", [2, 3])
-@pytest.mark.parametrize("mode,beta", [("allgather", 0.9), ("allgather", None), ("sharded", 0.9), ("push", 0.9)])
+@pytest.mark.parametrize("mode,beta", [("allgather", 0.9), ("allgather", None), ("sharded", 0.9), ("push", 0.9),
+                                       ("push-flags", 0.9)])
 def test_one_worker_per_gpu_over_nccl(world, mode, beta):
     if torch.cuda.device_count() < world:
         pytest.skip("needs %d GPUs, this machine shows %d: the one-worker-per-GPU path over NCCL is "

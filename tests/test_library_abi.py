@@ -38,6 +38,11 @@ def test_every_declared_symbol_is_exported(L):
     assert names == set(B.EXPORTS), "header and binding disagree on the entry points"
 
 
+def test_every_entry_point_has_its_argument_types_declared(L):
+    for n in B.EXPORTS:
+        assert getattr(L, n).argtypes is not None or n in ("ss_last_cuda_error",), "%s: argtypes not set" % n
+
+
 def test_packed_words(L):
     assert B.ss_packed_words(0) == 0
     assert B.ss_packed_words(1) == 1
@@ -150,6 +155,25 @@ def test_step_arguments_may_not_alias_what_the_step_writes(L):
     assert L.ss_fused_step(g, 0, (vp * 2)(0x50000, 0x10040), 2, 64, 0.9, 0, x, 0.1, 0.0, None, None) == B.SS_ERR_INVALID_ARG
     # the packed output of ss_signum_update on its momentum
     assert L.ss_signum_update(vp(0x10000), 0, vp(0x50000), 0.9, 64, vp(0x50010), None) == B.SS_ERR_INVALID_ARG
+
+
+def test_flag_exchange_argument_errors(L):
+    vp = ctypes.c_void_p
+    fake, arr = vp(0x1000), (vp * 2)(0x1000, 0x2000)
+    assert L.ss_flags_wait(fake, 3, 1, B.SS_FLAGS_MAX_TIMEOUT_NS + 1, fake, None) == B.SS_ERR_INVALID_ARG  # no long waits
+    assert L.ss_flags_wait(fake, 0, 1, 1000, fake, None) == B.SS_ERR_INVALID_ARG
+    assert L.ss_flags_wait(fake, 65, 1, 1000, fake, None) == B.SS_ERR_INVALID_ARG
+    assert L.ss_flags_wait(None, 3, 1, 1000, fake, None) == B.SS_ERR_INVALID_ARG
+    assert L.ss_flags_wait(fake, 3, 1, 1000, None, None) == B.SS_ERR_INVALID_ARG
+    assert L.ss_flags_wait(vp(0x1002), 3, 1, 1000, fake, None) == B.SS_ERR_MISALIGNED
+    assert L.ss_flags_signal(None, 2, 0, 1, None) == B.SS_ERR_INVALID_ARG
+    assert L.ss_flags_signal(arr, 0, 0, 1, None) == B.SS_ERR_INVALID_ARG
+    assert L.ss_flags_signal(arr, 65, 0, 1, None) == B.SS_ERR_INVALID_ARG
+    assert L.ss_flags_signal(arr, 2, 64, 1, None) == B.SS_ERR_INVALID_ARG
+    assert L.ss_flags_signal((vp * 2)(0x1000, None), 2, 0, 1, None) == B.SS_ERR_INVALID_ARG
+    assert L.ss_flags_signal((vp * 2)(0x1000, 0x2001), 2, 0, 1, None) == B.SS_ERR_MISALIGNED
+    assert L.ss_vote_apply_guarded(arr, 2, 64, 0, vp(0x70000), 0.1, 0.0, None, None, None) == B.SS_ERR_INVALID_ARG
+    assert L.ss_vote_apply_guarded(arr, 2, 64, 0, vp(0x70000), 0.1, 0.0, None, vp(0x9001), None) == B.SS_ERR_MISALIGNED
 
 
 def test_launch_option_validation(L):
