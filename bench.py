@@ -281,7 +281,7 @@ def entry_bytes(case, entry: str) -> int:
     mom = case.beta is not None
     if entry == "pack":
         return gb * d + wb
-    if entry == "signum_update":
+    if entry in ("signum_update", "signum_update_push"):
         return (gb + 8) * d + wb
     if entry == "vote":
         return (M + 1) * wb
@@ -410,6 +410,8 @@ def table_mode(args) -> None:
                 B.ss_sign_pack(grads[m], packed[m], stream)
             elif entry == "signum_update":
                 B.ss_signum_update(grads[m], moms[m], beta, packed[m], stream)
+            elif entry == "signum_update_push":      # one destination: the same bytes as signum_update
+                B.ss_signum_update_push(grads[m], moms[m], beta, [packed[m]], stream)
             elif entry == "vote":
                 B.ss_majority_vote(packed, case.d, case.flip_mask, vote, stream)
             elif entry == "apply":
@@ -457,7 +459,7 @@ def table_mode(args) -> None:
             stream.wait_stream(side)
 
         for entry in entries:
-            if entry == "signum_update" and not mom:
+            if entry in ("signum_update", "signum_update_push") and not mom:
                 continue
             ms = time_launches(lambda: call(entry), args.steps, max(3, args.warmup), stream, flush)
             nbytes = entry_bytes(case, entry)

@@ -231,10 +231,9 @@ def ss_vote_apply(packed: Sequence[torch.Tensor], param: torch.Tensor, lr: float
                                w_ptr, _stream(stream)), "ss_vote_apply")
 
 
-def ss_fused_step(grads: Sequence[torch.Tensor], momenta: Optional[Sequence[torch.Tensor]],
-                  param: torch.Tensor, beta: float, lr: float, weight_decay: float = 0.0,
-                  flip_mask: int = 0, vote_words_out: Optional[torch.Tensor] = None,
-                  stream=None) -> None:
+def _step_args(grads, momenta, param, vote_words_out):
+    """Marshalling shared by the fused-step entry points: (dtype code, gradient pointer array,
+    momentum pointer array or None, vote pointer or None, M, d)."""
     M = len(grads)
     d = param.numel()
     codes = {_dtype_code(g) for g in grads}
@@ -247,7 +246,15 @@ def ss_fused_step(grads: Sequence[torch.Tensor], momenta: Optional[Sequence[torc
             raise ValueError("need one momentum buffer per worker")
         v_arr = _ptr_array([_dev(v, torch.float32, "momenta[%d]" % m, d) for m, v in enumerate(momenta)])
     w_ptr = None if vote_words_out is None else _words(vote_words_out, d, "vote_words_out")
-    _check(lib().ss_fused_step(_ptr_array(g_ptrs), codes.pop(), v_arr, M, d, float(beta),
+    return codes.pop(), _ptr_array(g_ptrs), v_arr, w_ptr, M, d
+
+
+def ss_fused_step(grads: Sequence[torch.Tensor], momenta: Optional[Sequence[torch.Tensor]],
+                  param: torch.Tensor, beta: float, lr: float, weight_decay: float = 0.0,
+                  flip_mask: int = 0, vote_words_out: Optional[torch.Tensor] = None,
+                  stream=None) -> None:
+    code, g_arr, v_arr, w_ptr, M, d = _step_args(grads, momenta, param, vote_words_out)
+    _check(lib().ss_fused_step(g_arr, code, v_arr, M, d, float(beta),
                                int(flip_mask), _dev(param, torch.float32, "param"), float(lr),
                                float(weight_decay), w_ptr, _stream(stream)), "ss_fused_step")
 
@@ -279,19 +286,8 @@ def ss_fused_step_segments(grads: Sequence[torch.Tensor], momenta: Optional[Sequ
                            param: torch.Tensor, beta: float, segments_dev: torch.Tensor,
                            n_segments: int, flip_mask: int = 0,
                            vote_words_out: Optional[torch.Tensor] = None, stream=None) -> None:
-    M = len(grads)
-    d = param.numel()
-    codes = {_dtype_code(g) for g in grads}
-    if len(codes) != 1:
-        raise TypeError("all gradients must share one dtype")
-    g_ptrs = [_dev(g, None, "grads[%d]" % m, d) for m, g in enumerate(grads)]
-    v_arr = None
-    if momenta is not None:
-        if len(momenta) != M:
-            raise ValueError("need one momentum buffer per worker")
-        v_arr = _ptr_array([_dev(v, torch.float32, "momenta[%d]" % m, d) for m, v in enumerate(momenta)])
-    w_ptr = None if vote_words_out is None else _words(vote_words_out, d, "vote_words_out")
-    _check(lib().ss_fused_step_segments(_ptr_array(g_ptrs), codes.pop(), v_arr, M, d, float(beta),
+    code, g_arr, v_arr, w_ptr, M, d = _step_args(grads, momenta, param, vote_words_out)
+    _check(lib().ss_fused_step_segments(g_arr, code, v_arr, M, d, float(beta),
                                         int(flip_mask), _dev(param, torch.float32, "param"),
                                         _segments(segments_dev, n_segments), int(n_segments), w_ptr,
                                         _stream(stream)), "ss_fused_step_segments")
@@ -318,11 +314,9 @@ def ss_apply_vote_segments(param: torch.Tensor, vote_words: torch.Tensor, segmen
                                         _stream(stream)), "ss_apply_vote_segments")
 
 
-def ss_fused_step_host(host_grads: Sequence[torch.Tensor], staging: Sequence[torch.Tensor],
-                       momenta: Optional[Sequence[torch.Tensor]], param: torch.Tensor, beta: float,
-                       lr: float, weight_decay: float, flip_mask: int,
-                       vote_words_dev: torch.Tensor, host_vote_out: Optional[torch.Tensor],
-                       stream=None) -> None:
+def _host_step_args(host_grads, momenta, param, host_vote_out):
+    """Marshalling shared by the two host-gradient entry points: (dtype code, host pointer array,
+    momentum pointer array or None, host vote pointer or None, M, d)."""
     M = len(host_grads)
     d = param.numel()
     codes = {_dtype_code(g) for g in host_grads}
@@ -333,9 +327,6 @@ def ss_fused_step_host(host_grads: Sequence[torch.Tensor], staging: Sequence[tor
         if g.is_cuda or g.dim() != 1 or not g.is_contiguous() or g.numel() != d:
             raise ValueError("host_grads[%d] must be a contiguous 1-D host tensor of d elements" % m)
         h_ptrs.append(g.data_ptr())
-    if len(staging) != M:
-        raise ValueError("need one staging buffer per worker")
-    s_ptrs = [_dev(s, host_grads[0].dtype, "staging[%d]" % m, d) for m, s in enumerate(staging)]
     v_arr = None
     if momenta is not None:
         if len(momenta) != M:
@@ -347,7 +338,19 @@ def ss_fused_step_host(host_grads: Sequence[torch.Tensor], staging: Sequence[tor
                 or host_vote_out.numel() != ss_packed_words(d) or not host_vote_out.is_contiguous()):
             raise ValueError("host_vote_out must be a contiguous host int32 tensor of ceil(d/32) words")
         hv = host_vote_out.data_ptr()
-    _check(lib().ss_fused_step_host(_ptr_array(h_ptrs), codes.pop(), _ptr_array(s_ptrs), v_arr, M, d,
+    return codes.pop(), _ptr_array(h_ptrs), v_arr, hv, M, d
+
+
+def ss_fused_step_host(host_grads: Sequence[torch.Tensor], staging: Sequence[torch.Tensor],
+                       momenta: Optional[Sequence[torch.Tensor]], param: torch.Tensor, beta: float,
+                       lr: float, weight_decay: float, flip_mask: int,
+                       vote_words_dev: torch.Tensor, host_vote_out: Optional[torch.Tensor],
+                       stream=None) -> None:
+    code, h_arr, v_arr, hv, M, d = _host_step_args(host_grads, momenta, param, host_vote_out)
+    if len(staging) != M:
+        raise ValueError("need one staging buffer per worker")
+    s_ptrs = [_dev(s, host_grads[0].dtype, "staging[%d]" % m, d) for m, s in enumerate(staging)]
+    _check(lib().ss_fused_step_host(h_arr, code, _ptr_array(s_ptrs), v_arr, M, d,
                                     float(beta), int(flip_mask), _dev(param, torch.float32, "param"),
                                     float(lr), float(weight_decay),
                                     _words(vote_words_dev, d, "vote_words_dev"), hv, _stream(stream)),
@@ -362,29 +365,10 @@ def ss_fused_step_host_static(host_grads: Sequence[torch.Tensor],
     """ss_fused_step_host for callers that may not allocate device memory: the gradients are
     staged in a fixed array inside the library (at most SS_STATIC_STAGING_BYTES for all M workers
     together), so no staging tensors are passed. The first call on a device looks up that array's
-    address; make it during start-up. Calls that overlap on the GPU race on the array."""
-    M = len(host_grads)
-    d = param.numel()
-    codes = {_dtype_code(g) for g in host_grads}
-    if len(codes) != 1:
-        raise TypeError("all gradients must share one dtype")
-    h_ptrs = []
-    for m, g in enumerate(host_grads):
-        if g.is_cuda or g.dim() != 1 or not g.is_contiguous() or g.numel() != d:
-            raise ValueError("host_grads[%d] must be a contiguous 1-D host tensor of d elements" % m)
-        h_ptrs.append(g.data_ptr())
-    v_arr = None
-    if momenta is not None:
-        if len(momenta) != M:
-            raise ValueError("need one momentum buffer per worker")
-        v_arr = _ptr_array([_dev(v, torch.float32, "momenta[%d]" % m, d) for m, v in enumerate(momenta)])
-    hv = None
-    if host_vote_out is not None:
-        if (host_vote_out.is_cuda or host_vote_out.dtype != torch.int32
-                or host_vote_out.numel() != ss_packed_words(d) or not host_vote_out.is_contiguous()):
-            raise ValueError("host_vote_out must be a contiguous host int32 tensor of ceil(d/32) words")
-        hv = host_vote_out.data_ptr()
-    _check(lib().ss_fused_step_host_static(_ptr_array(h_ptrs), codes.pop(), v_arr, M, d, float(beta),
+    address (and, with lazy module loading, is what reserves the array); make it during start-up.
+    Calls that overlap on the GPU race on the array."""
+    code, h_arr, v_arr, hv, M, d = _host_step_args(host_grads, momenta, param, host_vote_out)
+    _check(lib().ss_fused_step_host_static(h_arr, code, v_arr, M, d, float(beta),
                                            int(flip_mask), _dev(param, torch.float32, "param"),
                                            float(lr), float(weight_decay),
                                            _words(vote_words_dev, d, "vote_words_dev"), hv,
