@@ -790,6 +790,13 @@ def worker_per_gpu_mode(args) -> None:
     kernel_ms = sharding.max_over_ranks(kernel_ms, dev)
     exchange_ms = sharding.max_over_ranks(exchange_ms, dev)
     ms_step = ms_total / args.steps
+    # Algorithm 1 keeps one copy of x per worker and every worker applies the same vote: after any
+    # number of steps all replicas must hold the same bits. Compare a digest of x across the ranks.
+    digest = torch.stack([x.view(torch.int32).sum(dtype=torch.int64),
+                          (x.view(torch.int32)[::97].to(torch.int64) * 31).sum()])
+    digests = [torch.zeros_like(digest) for _ in range(world)]
+    dist.all_gather(digests, digest)
+    replicas_agree = all(bool(torch.equal(t, digests[0])) for t in digests)
     if rank == 0:
         W4 = ((case.d + 31) // 32) * 4
         paper_bits = 2 * world * case.d                      # Appendix B: 2 M d bits per iteration, whole system
@@ -808,12 +815,15 @@ def worker_per_gpu_mode(args) -> None:
             "bytes_received_sharded_formula": 2 * (world - 1) * W4 // world,
             "paper_bits_per_iteration_whole_system": paper_bits,
             "gpu_launches": launches_per_step * args.steps,
+            "replicas_agree": replicas_agree,
             "note": ("M = number of ranks: every rank is one worker of Algorithm 1 with its own replica of x; "
                      "params/s counts the d parameters once"),
         }
         line.update(spread(per_step))
         print(json.dumps(line), flush=True)
     dist.destroy_process_group()
+    if not replicas_agree:
+        raise SystemExit("worker-per-gpu: the workers' copies of x differ after %d steps" % (args.steps + args.warmup))
 
 
 def main() -> None:

@@ -4,8 +4,9 @@ TEST INFRASTRUCTURE ONLY: the slow, plain CPU definition the CUDA library is che
 against. Nothing on the product path imports this package; only the tests, the smoke
 check and the benchmark's CPU-baseline leg do. It shares no code with the CUDA path.
 
-The arithmetic lives in ``signsgd_oracle.cpp`` (plain C++, one coordinate at a time);
-this module only compiles it with g++ on first use, loads it with ctypes and passes
+The arithmetic lives in ``signsgd_oracle.cpp`` (Algorithm 1) and ``ternary_oracle.cpp`` (the
+comparison codec of Appendix B), plain C++, one coordinate at a time; this module only compiles
+them with g++ on first use, loads it with ctypes and passes
 numpy arrays through. Arrays: gradients ``float32`` or raw bf16 bit patterns as
 ``uint16``; momenta and parameters ``float32`` (updated in place); packed signs and
 votes ``uint32`` with ``ceil(d/32)`` words, coordinate ``32 j + i`` at bit ``i`` of word ``j``.

@@ -22,28 +22,46 @@ struct Draw4 {
     uint32_t r[4];
 };
 
-__device__ __forceinline__ Draw4 philox4x32_10(uint64_t block, uint64_t seed) {
+// The ten round keys of a seed (key + round * Weyl constants), formed once on the host and
+// handed to the kernel as parameters: the generator then costs four multiplies and two
+// three-input XORs per round and no key arithmetic.
+struct PhiloxKeys {
+    uint32_t k0[10], k1[10];
+};
+
+inline PhiloxKeys philox_keys(uint64_t seed) {
+    PhiloxKeys k;
+    uint32_t a = static_cast<uint32_t>(seed), b = static_cast<uint32_t>(seed >> 32);
+    for (int round = 0; round < 10; ++round) {
+        k.k0[round] = a;
+        k.k1[round] = b;
+        a += 0x9E3779B9u;
+        b += 0xBB67AE85u;
+    }
+    return k;
+}
+
+__device__ __forceinline__ Draw4 philox4x32_10(uint64_t block, const PhiloxKeys& key) {
     uint32_t c0 = static_cast<uint32_t>(block), c1 = static_cast<uint32_t>(block >> 32), c2 = 0u, c3 = 0u;
-    uint32_t k0 = static_cast<uint32_t>(seed), k1 = static_cast<uint32_t>(seed >> 32);
 #pragma unroll
     for (int round = 0; round < 10; ++round) {
         const uint32_t hi0 = __umulhi(0xD2511F53u, c0), lo0 = 0xD2511F53u * c0;
         const uint32_t hi1 = __umulhi(0xCD9E8D57u, c2), lo1 = 0xCD9E8D57u * c2;
-        const uint32_t n0 = hi1 ^ c1 ^ k0, n2 = hi0 ^ c3 ^ k1;
+        const uint32_t n0 = hi1 ^ c1 ^ key.k0[round], n2 = hi0 ^ c3 ^ key.k1[round];
         c0 = n0, c1 = lo1, c2 = n2, c3 = lo0;
-        k0 += 0x9E3779B9u;
-        k1 += 0xBB67AE85u;
     }
     return Draw4{{c0, c1, c2, c3}};
 }
 
 // Two-bit code of one coordinate: kept iff RN(u * gmax) < |g| with u = (r >> 9) * 2^-23, i.e.
 // with probability |g| / gmax to within 2^-23; 1 = +1, 3 = -1, 0 = dropped (also NaN, and every
-// coordinate when gmax is 0 or Inf). u is formed without an integer-to-float conversion (a
-// quarter-rate instruction): the 23 bits become the mantissa of a float in [1, 2), minus 1, exact.
+// coordinate when gmax is 0 or Inf). The 23 bits become the mantissa of a float f in [1, 2), so
+// u = f - 1 exactly and needs no integer-to-float conversion, and RN((f - 1) * gmax) is formed by
+// one fused multiply-add, f * gmax - gmax: the exact value is the same and it is rounded once.
+// (For gmax = Inf the fused form gives NaN where the product gives Inf; neither is < |g|.)
 __device__ __forceinline__ uint32_t ternary_code(float g, uint32_t r, float gmax) {
-    const float u = __fsub_rn(__uint_as_float(0x3F800000u | (r >> 9)), 1.0f);
-    const bool kept = __fmul_rn(u, gmax) < fabsf(g);
+    const float f = __uint_as_float(0x3F800000u | (r >> 9));
+    const bool kept = __fmaf_rn(f, gmax, -gmax) < fabsf(g);
     return kept ? (g < 0.0f ? 3u : 1u) : 0u;
 }
 
@@ -79,7 +97,7 @@ __global__ void __launch_bounds__(256) absmax_kernel(const void* __restrict__ g,
 template <typename GT, bool VEC>
 __global__ void __launch_bounds__(256)
 ternary_pack_kernel(const void* __restrict__ g, int64_t d, const float* __restrict__ gmax_dev,
-                    uint64_t seed, uint32_t* __restrict__ codes) {
+                    const __grid_constant__ PhiloxKeys seed, uint32_t* __restrict__ codes) {
     const float gmax = __ldg(gmax_dev);
     const int lane = threadIdx.x & 31;
     const int k4 = lane & 3;
@@ -153,8 +171,7 @@ inline bool ranges_overlap(const void* p, size_t n, const void* q, size_t m) {
     return n != 0 && m != 0 && a < b + m && b < a + n;
 }
 
-template <typename Kernel>
-cudaError_t stream_grid(Kernel kernel, int threads, int64_t items, int per_sm, int* grid) {
+inline cudaError_t stream_grid(int threads, int64_t items, int per_sm, int* grid) {
     // grid-stride kernels: enough blocks to cover the items, at most per_sm blocks per SM
     cudaError_t err = cudaSuccess;
     const int sms = device_sm_count(&err);
@@ -164,7 +181,6 @@ cudaError_t stream_grid(Kernel kernel, int threads, int64_t items, int per_sm, i
     if (blocks > cap) blocks = cap;
     if (blocks < 1) blocks = 1;
     *grid = static_cast<int>(blocks);
-    (void)kernel;
     return cudaSuccess;
 }
 
@@ -196,7 +212,7 @@ int ss_absmax(const void* grad, ss_dtype dt, int64_t d, float* absmax_dev, void*
     const int64_t items = vec ? ((d >> 2) + 1) / 2 + 4 : d;
 #define SS_ABSMAX(GT, VEC)                                                        \
     do {                                                                          \
-        e = stream_grid(absmax_kernel<GT, VEC>, threads, items, 16, &grid);       \
+        e = stream_grid(threads, items, 16, &grid);                               \
         if (e != cudaSuccess) return cuda_status_public(e);                       \
         absmax_kernel<GT, VEC><<<grid, threads, 0, st>>>(grad, d, out);           \
     } while (0)
@@ -225,11 +241,12 @@ int ss_ternary_pack(const void* grad, ss_dtype dt, int64_t d, const float* absma
     int grid = 1;
     cudaError_t e;
     const int64_t quads = ((d >> 4) << 2);
+    const PhiloxKeys keys = philox_keys(seed);
 #define SS_TPACK(GT, VEC)                                                                  \
     do {                                                                                   \
         e = pick_grid(ternary_pack_kernel<GT, VEC>, threads, (quads + threads - 1) / threads, &grid); \
         if (e != cudaSuccess) return cuda_status_public(e);                                \
-        ternary_pack_kernel<GT, VEC><<<grid, threads, 0, st>>>(grad, d, absmax_dev, seed, out_codes); \
+        ternary_pack_kernel<GT, VEC><<<grid, threads, 0, st>>>(grad, d, absmax_dev, keys, out_codes); \
     } while (0)
     if (dt == SS_F32) {
         if (vec) SS_TPACK(F32, true); else SS_TPACK(F32, false);

@@ -125,6 +125,7 @@ def test_worker_per_gpu_mode_runs_on_one_rank(layout):
     assert r["config"]["M"] == 1 and r["value"] > 0 and r["ms_per_step"] > 0
     assert r["kernel_ms_per_step"] > 0 and r["exchange_ms_per_step"] >= 0
     assert r["kernel_ms_per_step"] + r["exchange_ms_per_step"] <= r["ms_per_step"] * 1.05
+    assert r["replicas_agree"] is True
     assert r["bytes_received_per_worker_per_step"] == 0          # a lone worker receives nothing
     assert r["paper_bits_per_iteration_whole_system"] == 2 * 1000008
     per_step = 3 if extra else {"allgather": 2, "sharded": 3, "push": 2}[layout]
