@@ -310,6 +310,13 @@ int ss_vote_apply_guarded(const uint32_t* const* packed, int M, int64_t d, uint6
                           const uint32_t* skip_if_nonzero_dev, void* cuda_stream) {
     if (skip_if_nonzero_dev == nullptr) return SS_ERR_INVALID_ARG;
     if (!aligned(skip_if_nonzero_dev, 4)) return SS_ERR_MISALIGNED;
+    if (d > 0 && d_ok(d)) {  // the guard word is read while the call writes: it may lie in neither output
+        if (param != nullptr && overlap(skip_if_nonzero_dev, 4, param, static_cast<size_t>(d) * 4))
+            return SS_ERR_INVALID_ARG;
+        if (vote_words_out != nullptr &&
+            overlap(skip_if_nonzero_dev, 4, vote_words_out, static_cast<size_t>((d + 31) / 32) * 4))
+            return SS_ERR_INVALID_ARG;
+    }
     return vote_apply_common(packed, M, d, flip_mask, param, lr, weight_decay, nullptr, 0,
                              vote_words_out, cuda_stream, skip_if_nonzero_dev);
 }

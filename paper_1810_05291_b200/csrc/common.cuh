@@ -9,21 +9,56 @@
 
 namespace ss {
 
+// Load policies of the streaming kernels. Every byte is touched once, so the natural form is the
+// evict-first load (ld.global.cs), and it is the better one for pure read streams (sign packing,
+// packed words). In the step kernels, which also write, plain loads (cached at all levels) measure
+// faster: same box, same run, fused step, ms per launch, evict-first everywhere / plain for the
+// read-modify-write streams only (momenta, parameters) / plain everywhere:
+//   M = 15 fp32 Signum (ResNet-50 size)   0.7108 / 0.7034 / 0.6949
+//   M = 7 fp32 signSGD (AlexNet size)     0.3179 / 0.3175 / 0.3074
+//   M = 15 bf16 Signum, octet kernel      0.6063 / 0.5989 / 0.5940
+//   M = 15 fp32 signSGD, d = 2^28         2.6510 / 2.6504 / 2.5375
+// with two exceptions that keep evict-first gradient loads: the run-time-M kernel without
+// momentum (M = 63, d = 2^28: 10.1 ms either way, 18.2 ms with plain gradient loads) and the
+// one-worker bf16 momentum update, which keeps evict-first loads throughout (0.0389 against
+// 0.0410 ms). The kernels therefore take the policy of their gradient loads as a compile-time
+// flag; momenta and parameters are loaded plain (ld_rmw) everywhere else.
+template <typename T>
+__device__ __forceinline__ T ld_stream(const T* p) {
+    return __ldcs(p);
+}
+template <bool PLAIN, typename T>
+__device__ __forceinline__ T ld_grad(const T* p) {
+    if constexpr (PLAIN) return *p;
+    else return __ldcs(p);
+}
+template <typename T>
+__device__ __forceinline__ T ld_rmw(const T* p) {
+    return *p;
+}
+template <bool PLAIN, typename T>
+__device__ __forceinline__ T ld_rmw_as(const T* p) {  // for the one kernel that keeps evict-first throughout
+    if constexpr (PLAIN) return *p;
+    else return __ldcs(p);
+}
+
 struct F32 {
     static constexpr int kBytes = 4;
     // four consecutive coordinates starting at coordinate 4 q
+    template <bool PLAIN = false>
     static __device__ __forceinline__ float4 load4(const void* base, int64_t q) {
-        return __ldcs(reinterpret_cast<const float4*>(base) + q);
+        return ld_grad<PLAIN>(reinterpret_cast<const float4*>(base) + q);
     }
     static __device__ __forceinline__ float load1(const void* base, int64_t c) {
-        return __ldcs(reinterpret_cast<const float*>(base) + c);
+        return ld_stream(reinterpret_cast<const float*>(base) + c);
     }
 };
 
 struct BF16 {
     static constexpr int kBytes = 2;
+    template <bool PLAIN = false>
     static __device__ __forceinline__ float4 load4(const void* base, int64_t q) {
-        const uint2 r = __ldcs(reinterpret_cast<const uint2*>(base) + q);
+        const uint2 r = ld_grad<PLAIN>(reinterpret_cast<const uint2*>(base) + q);
         float4 f;
         f.x = __uint_as_float(r.x << 16);
         f.y = __uint_as_float(r.x & 0xFFFF0000u);
@@ -32,7 +67,7 @@ struct BF16 {
         return f;
     }
     static __device__ __forceinline__ float load1(const void* base, int64_t c) {
-        const unsigned short h = __ldcs(reinterpret_cast<const unsigned short*>(base) + c);
+        const unsigned short h = ld_stream(reinterpret_cast<const unsigned short*>(base) + c);
         return __uint_as_float(static_cast<uint32_t>(h) << 16);
     }
 };

@@ -77,7 +77,7 @@ __device__ __forceinline__ void step_word_ballot(const StepArgs<NP>& a, int64_t 
         for (int k = 0; k < NB; ++k) {
             const bool on = valid && (M_CT > 0 || m0 + k < M);
             gs[k] = on ? GT::load1(a.g[m0 + k < NP ? m0 + k : 0], c) : -1.0f;
-            if (MOM) vs[k] = on ? __ldcs(a.v[m0 + k < NP ? m0 + k : 0] + c) : 0.0f;
+            if (MOM) vs[k] = on ? ld_rmw(a.v[m0 + k < NP ? m0 + k : 0] + c) : 0.0f;
         }
         uint32_t w[NB];
 #pragma unroll
@@ -159,6 +159,8 @@ __global__ void __launch_bounds__(256)
 step_vec_kernel(const __grid_constant__ StepArgs<StepShape<M_CT, MOM>::NP> a) {
     using S = StepShape<M_CT, MOM>;
     constexpr int LB = S::LB, U = S::U;
+    // gradient loads: plain, except in the run-time-M kernel without momentum (see ld_grad)
+    constexpr bool G_PLAIN = M_CT > 0 || MOM;
     const int M = M_CT > 0 ? M_CT : a.M;
     const int lane = threadIdx.x & 31;
     const int64_t n_quads = (a.d >> 5) << 3;  // quads lying in complete words
@@ -177,7 +179,7 @@ step_vec_kernel(const __grid_constant__ StepArgs<StepShape<M_CT, MOM>::NP> a) {
             q[u] = base + static_cast<int64_t>(u) * blockDim.x + threadIdx.x;
             ok[u] = q[u] < n_quads;  // uniform over each 8-lane group: n_quads is a multiple of 8
             cnt[u].clear();
-            if (APPLY && ok[u]) xq[u] = __ldcs(reinterpret_cast<const float4*>(a.x) + q[u]);
+            if (APPLY && ok[u]) xq[u] = ld_rmw(reinterpret_cast<const float4*>(a.x) + q[u]);
         }
 
         auto batch = [&](int m0, auto nb_tag) {
@@ -189,9 +191,10 @@ step_vec_kernel(const __grid_constant__ StepArgs<StepShape<M_CT, MOM>::NP> a) {
                 for (int k = 0; k < NB; ++k) {
                     const bool on = ok[u] && (M_CT > 0 || m0 + k < M);
                     const int mi = m0 + k < S::NP ? m0 + k : 0;
-                    gq[u][k] = on ? GT::load4(a.g[mi], q[u]) : make_float4(-1.f, -1.f, -1.f, -1.f);
+                    gq[u][k] = on ? GT::template load4<G_PLAIN>(a.g[mi], q[u])
+                                  : make_float4(-1.f, -1.f, -1.f, -1.f);
                     if (MOM)
-                        vq[u][k] = on ? __ldcs(reinterpret_cast<const float4*>(a.v[mi]) + q[u])
+                        vq[u][k] = on ? ld_rmw(reinterpret_cast<const float4*>(a.v[mi]) + q[u])
                                       : make_float4(0.f, 0.f, 0.f, 0.f);
                 }
             }
@@ -310,7 +313,7 @@ pack_oct_bf16_kernel(const void* __restrict__ g, uint32_t* __restrict__ words, i
 #pragma unroll
         for (int u = 0; u < U; ++u) {
             const int64_t o = base + static_cast<int64_t>(u) * blockDim.x + threadIdx.x;
-            v[u] = o < n_oct ? __ldcs(reinterpret_cast<const uint4*>(g) + o)
+            v[u] = o < n_oct ? ld_stream(reinterpret_cast<const uint4*>(g) + o)
                              : make_uint4(0x80008000u, 0x80008000u, 0x80008000u, 0x80008000u);
         }
 #pragma unroll
@@ -423,8 +426,9 @@ signum_push_kernel(const void* __restrict__ g, float* __restrict__ v, float beta
         for (int u = 0; u < U; ++u) {
             const int64_t q = base + static_cast<int64_t>(u) * blockDim.x + threadIdx.x;
             const bool ok = q < n_quads;
-            gq[u] = ok ? GT::load4(g, q) : make_float4(-1.f, -1.f, -1.f, -1.f);
-            vq[u] = ok ? __ldcs(reinterpret_cast<const float4*>(v) + q) : make_float4(0.f, 0.f, 0.f, 0.f);
+            // fp32 gradients plain, bf16 (64-bit requests) evict-first: as measured for ss_signum_update
+            gq[u] = ok ? GT::template load4<GT::kBytes == 4>(g, q) : make_float4(-1.f, -1.f, -1.f, -1.f);
+            vq[u] = ok ? ld_rmw(reinterpret_cast<const float4*>(v) + q) : make_float4(0.f, 0.f, 0.f, 0.f);
         }
 #pragma unroll
         for (int u = 0; u < U; ++u) {
@@ -470,7 +474,7 @@ signum_push_ballot_kernel(const void* __restrict__ g, float* __restrict__ v, flo
         for (int k = 0; k < PACK_WORDS; ++k) {
             const int64_t c = ((j0 + k) << 5) + lane;
             gs[k] = c < d ? GT::load1(g, c) : -1.0f;
-            vs[k] = c < d ? __ldcs(v + c) : 0.0f;
+            vs[k] = c < d ? ld_rmw(v + c) : 0.0f;
         }
         uint32_t mine = 0u;
 #pragma unroll
@@ -536,7 +540,7 @@ single_worker_kernel(const void* __restrict__ g, float* __restrict__ x, uint32_t
             const int64_t q = base + static_cast<int64_t>(u) * blockDim.x + threadIdx.x;
             const bool ok = q < n_quads;
             gq[u] = ok ? GT::load4(g, q) : make_float4(-1.f, -1.f, -1.f, -1.f);
-            xq[u] = ok ? __ldcs(reinterpret_cast<const float4*>(x) + q) : make_float4(0.f, 0.f, 0.f, 0.f);
+            xq[u] = ok ? ld_rmw(reinterpret_cast<const float4*>(x) + q) : make_float4(0.f, 0.f, 0.f, 0.f);
         }
 #pragma unroll
         for (int u = 0; u < U; ++u) {

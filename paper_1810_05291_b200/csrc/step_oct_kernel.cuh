@@ -41,6 +41,8 @@ __global__ void __launch_bounds__(256)
 step_oct_bf16_kernel(const __grid_constant__ StepArgs<OctShape<M_CT, MOM>::NP> a) {
     using S = OctShape<M_CT, MOM>;
     constexpr int LB = S::LB, U = S::U;
+    // loads: plain in the fused step, evict-first throughout in the one-worker momentum update (see ld_grad)
+    constexpr bool G_PLAIN = APPLY;
     const int M = M_CT > 0 ? M_CT : a.M;
     const int lane = threadIdx.x & 31;
     const int k4 = lane & 3;
@@ -61,8 +63,8 @@ step_oct_bf16_kernel(const __grid_constant__ StepArgs<OctShape<M_CT, MOM>::NP> a
             ok[u] = o[u] < n_oct;  // uniform over each 4-lane group: n_oct is a multiple of 4
             cnt[u].clear();
             if (APPLY && ok[u]) {
-                xlo[u] = __ldcs(reinterpret_cast<const float4*>(a.x) + 2 * o[u]);
-                xhi[u] = __ldcs(reinterpret_cast<const float4*>(a.x) + 2 * o[u] + 1);
+                xlo[u] = ld_rmw(reinterpret_cast<const float4*>(a.x) + 2 * o[u]);
+                xhi[u] = ld_rmw(reinterpret_cast<const float4*>(a.x) + 2 * o[u] + 1);
             }
         }
 
@@ -76,12 +78,12 @@ step_oct_bf16_kernel(const __grid_constant__ StepArgs<OctShape<M_CT, MOM>::NP> a
                 for (int k = 0; k < NB; ++k) {
                     const bool on = ok[u] && (M_CT > 0 || m0 + k < M);
                     const int mi = m0 + k < S::NP ? m0 + k : 0;
-                    gq[u][k] = on ? __ldcs(reinterpret_cast<const uint4*>(a.g[mi]) + o[u])
+                    gq[u][k] = on ? ld_grad<G_PLAIN>(reinterpret_cast<const uint4*>(a.g[mi]) + o[u])
                                   : make_uint4(0x80008000u, 0x80008000u, 0x80008000u, 0x80008000u);
                     if (MOM) {
                         const float4* vp = reinterpret_cast<const float4*>(a.v[mi]) + 2 * o[u];
-                        vlo[u][k] = on ? __ldcs(vp) : make_float4(0.f, 0.f, 0.f, 0.f);
-                        vhi[u][k] = on ? __ldcs(vp + 1) : make_float4(0.f, 0.f, 0.f, 0.f);
+                        vlo[u][k] = on ? ld_rmw_as<G_PLAIN>(vp) : make_float4(0.f, 0.f, 0.f, 0.f);
+                        vhi[u][k] = on ? ld_rmw_as<G_PLAIN>(vp + 1) : make_float4(0.f, 0.f, 0.f, 0.f);
                     }
                 }
             }

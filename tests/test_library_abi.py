@@ -174,6 +174,8 @@ def test_flag_exchange_argument_errors(L):
     assert L.ss_flags_signal((vp * 2)(0x1000, 0x2001), 2, 0, 1, None) == B.SS_ERR_MISALIGNED
     assert L.ss_vote_apply_guarded(arr, 2, 64, 0, vp(0x70000), 0.1, 0.0, None, None, None) == B.SS_ERR_INVALID_ARG
     assert L.ss_vote_apply_guarded(arr, 2, 64, 0, vp(0x70000), 0.1, 0.0, None, vp(0x9001), None) == B.SS_ERR_MISALIGNED
+    assert L.ss_vote_apply_guarded(arr, 2, 64, 0, vp(0x70000), 0.1, 0.0, None, vp(0x70010), None) == B.SS_ERR_INVALID_ARG  # guard inside param
+    assert L.ss_vote_apply_guarded(arr, 2, 64, 0, vp(0x70000), 0.1, 0.0, vp(0x80000), vp(0x80004), None) == B.SS_ERR_INVALID_ARG  # guard inside the vote
 
 
 def test_launch_option_validation(L):
