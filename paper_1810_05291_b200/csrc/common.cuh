@@ -18,9 +18,10 @@ namespace ss {
 //   M = 7 fp32 signSGD (AlexNet size)     0.3179 / 0.3175 / 0.3074
 //   M = 15 bf16 Signum, octet kernel      0.6063 / 0.5989 / 0.5940
 //   M = 15 fp32 signSGD, d = 2^28         2.6510 / 2.6504 / 2.5375
-// with two exceptions that keep evict-first gradient loads: the run-time-M kernel without
-// momentum (M = 63, d = 2^28: 10.1 ms either way, 18.2 ms with plain gradient loads) and the
-// one-worker bf16 momentum update, which keeps evict-first loads throughout (0.0389 against
+// with exceptions that keep evict-first gradient loads: the run-time-M kernel without momentum
+// (M = 63, d = 2^28: 10.1 ms either way, 18.2 ms with plain gradient loads), calls without
+// momentum that read less than 1.5 GiB of gradients (the launcher decides, step_kernel.cuh), and
+// the one-worker bf16 momentum update, which keeps evict-first loads throughout (0.0389 against
 // 0.0410 ms). The kernels therefore take the policy of their gradient loads as a compile-time
 // flag; momenta and parameters are loaded plain (ld_rmw) everywhere else.
 template <typename T>

@@ -154,13 +154,12 @@ __device__ __forceinline__ void store_words(uint32_t* words, const uint32_t* nib
     }
 }
 
-template <int M_CT, typename GT, bool MOM, bool APPLY, bool SEG>
+// G_PLAIN: policy of the gradient loads (see ld_grad), chosen by the launcher.
+template <int M_CT, typename GT, bool MOM, bool APPLY, bool SEG, bool G_PLAIN>
 __global__ void __launch_bounds__(256)
 step_vec_kernel(const __grid_constant__ StepArgs<StepShape<M_CT, MOM>::NP> a) {
     using S = StepShape<M_CT, MOM>;
     constexpr int LB = S::LB, U = S::U;
-    // gradient loads: plain, except in the run-time-M kernel without momentum (see ld_grad)
-    constexpr bool G_PLAIN = M_CT > 0 || MOM;
     const int M = M_CT > 0 ? M_CT : a.M;
     const int lane = threadIdx.x & 31;
     const int64_t n_quads = (a.d >> 5) << 3;  // quads lying in complete words
@@ -604,6 +603,8 @@ void fill_step_args(StepArgs<NP>& a, const StepDesc& s, bool mom) {
     a.n_seg = s.n_seg;
 }
 
+constexpr int64_t kPlainFromBytes = int64_t(3) << 29;  // 1.5 GiB of gradients per call
+
 template <int M_CT, typename GT, bool MOM, bool APPLY, bool VEC, bool SEG = false>
 cudaError_t launch_step_inst(const StepDesc& s, cudaStream_t st) {
     using S = StepShape<M_CT, MOM>;
@@ -613,12 +614,28 @@ cudaError_t launch_step_inst(const StepDesc& s, cudaStream_t st) {
     int grid = 1;
     cudaError_t err;
     if constexpr (VEC) {
-        auto kernel = step_vec_kernel<M_CT, GT, MOM, APPLY, SEG>;
         const int64_t quads = (s.d >> 5) << 3;
         const int64_t tile = static_cast<int64_t>(threads) * S::U;
-        err = pick_grid(kernel, threads, (quads + tile - 1) / tile, &grid);
+        err = pick_grid(step_vec_kernel<M_CT, GT, MOM, APPLY, SEG, false>, threads, (quads + tile - 1) / tile, &grid);
         if (err != cudaSuccess) return err;
-        kernel<<<grid, threads, 0, st>>>(a);
+        // Gradient loads (see ld_grad): plain with momentum; evict-first in the run-time-M kernel
+        // without momentum; in the unrolled kernels without momentum plain once the call reads
+        // kPlainFromBytes of gradients or more. Measured plain / evict-first, fp32, isolated
+        // launches: M = 15: 1.02 at d = 2^24 (1.0 GB), 1.00 at 25.6 M (1.5 GB), 0.97 at 2^26, 0.96
+        // at 2^28; M = 7: 1.05 at 2^24 (0.5 GB), 0.97 at 2^26 (1.9 GB) and at 61 M; M = 3: 1.13 at
+        // 2^24, 1.02 at 2^26 (0.8 GB), 0.95 at 2^28 (3.2 GB).
+        bool plain = MOM;
+        if constexpr (!MOM && M_CT > 0)
+            plain = static_cast<int64_t>(s.M) * s.d * GT::kBytes >= kPlainFromBytes;
+        if constexpr (MOM) {
+            step_vec_kernel<M_CT, GT, MOM, APPLY, SEG, true><<<grid, threads, 0, st>>>(a);
+        } else if constexpr (M_CT == 0) {
+            step_vec_kernel<M_CT, GT, MOM, APPLY, SEG, false><<<grid, threads, 0, st>>>(a);
+        } else if (plain) {
+            step_vec_kernel<M_CT, GT, MOM, APPLY, SEG, true><<<grid, threads, 0, st>>>(a);
+        } else {
+            step_vec_kernel<M_CT, GT, MOM, APPLY, SEG, false><<<grid, threads, 0, st>>>(a);
+        }
     } else {
         auto kernel = step_ballot_kernel<M_CT, GT, MOM, APPLY, SEG>;
         const int64_t W = (s.d + 31) >> 5;
