@@ -43,10 +43,10 @@ NOMINAL_HBM_GBS = 8000.0
 # sources have changed since, the entry no longer describes the kernel that runs and
 # roofline.traffic is reported as null until the counters are taken again.
 NCU_DRAM_BYTES_PER_COORD = {
-    (15, 4, True): {"bytes_per_coord": (1.040214e9 + 486.63e6) / 8388608, "capture_d": 8388608,
-                    "sources": "f32", "source_hash": "48a87cc755c30efc"},
-    (15, 2, True): {"bytes_per_coord": (788.562e6 + 483.48e6) / 8388608, "capture_d": 8388608,
-                    "sources": "bf16", "source_hash": "f2f115cf80595fd9"},
+    (15, 4, True): {"bytes_per_coord": (1.040214e9 + 486.57e6) / 8388608, "capture_d": 8388608,
+                    "sources": "f32", "source_hash": "5e92bc2105780016"},
+    (15, 2, True): {"bytes_per_coord": (788.560e6 + 483.18e6) / 8388608, "capture_d": 8388608,
+                    "sources": "bf16", "source_hash": "fcf6dbe2805715df"},
 }
 KERNEL_SOURCES = {
     "f32": ("step_kernel.cuh", "bitslice.cuh", "common.cuh"),

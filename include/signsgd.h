@@ -372,12 +372,16 @@ int ss_ternary_unpack(const uint32_t* codes, int64_t d, const float* scale_dev, 
 
 /*
  * Launch-shape override for benchmarking sweeps: not part of the method, and the one piece of
- * process-wide state in the library (two integers, written and read atomically; a launch uses the
+ * process-wide state in the library (three integers, written and read atomically; a launch uses the
  * values it finds when it is made, so change them only between calls whose shape matters).
  *   key: "threads" (block size: a multiple of 32 in [64, 256], the bound the kernels are compiled
  *        for; 0 = default, 256) or
  *        "blocks_per_sm" (0 = one block per tile, the default; n > 0 = a persistent grid of
- *        n blocks per SM that strides over the tiles; at most 4096).
+ *        n blocks per SM that strides over the tiles; at most 4096) or
+ *        "plain_loads_from_mib" (ss_fused_step without momentum: the gradient bytes of a call, in
+ *        MiB, from which the gradients are fetched with plain loads instead of evict-first ones;
+ *        0 = default, 1536; 1 = practically always; at most 2^20 = never). Results do not depend
+ *        on any of the three.
  * Returns SS_ERR_INVALID_ARG for an unknown key or a value out of range.
  */
 int ss_set_launch_option(const char* key, int value);

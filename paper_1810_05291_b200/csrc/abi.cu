@@ -11,6 +11,8 @@ namespace ss {
 namespace {
 std::atomic<int> g_opt_threads{0};
 std::atomic<int> g_opt_blocks_per_sm{0};
+std::atomic<int> g_opt_plain_from_mib{0};
+constexpr int kDefaultPlainFromMib = 1536;
 }  // namespace
 
 int launch_threads() {
@@ -19,6 +21,11 @@ int launch_threads() {
 }
 
 int launch_blocks_per_sm() { return g_opt_blocks_per_sm.load(std::memory_order_relaxed); }
+
+int64_t launch_plain_loads_from_bytes() {
+    const int mib = g_opt_plain_from_mib.load(std::memory_order_relaxed);
+    return static_cast<int64_t>(mib > 0 ? mib : kDefaultPlainFromMib) << 20;
+}
 
 int device_sm_count(cudaError_t* err) {
     static int cached[64] = {0};
@@ -163,6 +170,11 @@ int ss_set_launch_option(const char* key, int value) {
         if (value != 0 && (value < 64 || value > kMaxBlockThreads || (value & 31) != 0))
             return SS_ERR_INVALID_ARG;
         g_opt_threads.store(value, std::memory_order_relaxed);
+        return SS_OK;
+    }
+    if (std::strcmp(key, "plain_loads_from_mib") == 0) {
+        if (value < 0 || value > (1 << 20)) return SS_ERR_INVALID_ARG;
+        g_opt_plain_from_mib.store(value, std::memory_order_relaxed);
         return SS_OK;
     }
     if (std::strcmp(key, "blocks_per_sm") == 0) {

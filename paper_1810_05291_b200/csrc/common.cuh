@@ -158,6 +158,8 @@ __device__ __forceinline__ float4 update_seg4(const ss_segment* seg, int n, int6
 constexpr int kMaxBlockThreads = 256;  // every kernel is compiled with __launch_bounds__(256)
 int launch_threads();        // block size to use: the "threads" option, or 256 when it is 0
 int launch_blocks_per_sm();  // 0: one block per tile; > 0: persistent grid of this many blocks per SM
+int64_t launch_plain_loads_from_bytes();  // gradient bytes per call from which the unrolled kernels
+                                          // without momentum load the gradients plain (see ld_grad)
 int device_sm_count(cudaError_t* err);
 
 // Grid size for a grid-stride kernel. Default: one block per tile. On B200 the hardware block

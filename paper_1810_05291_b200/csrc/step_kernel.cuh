@@ -603,8 +603,6 @@ void fill_step_args(StepArgs<NP>& a, const StepDesc& s, bool mom) {
     a.n_seg = s.n_seg;
 }
 
-constexpr int64_t kPlainFromBytes = int64_t(3) << 29;  // 1.5 GiB of gradients per call
-
 template <int M_CT, typename GT, bool MOM, bool APPLY, bool VEC, bool SEG = false>
 cudaError_t launch_step_inst(const StepDesc& s, cudaStream_t st) {
     using S = StepShape<M_CT, MOM>;
@@ -620,13 +618,14 @@ cudaError_t launch_step_inst(const StepDesc& s, cudaStream_t st) {
         if (err != cudaSuccess) return err;
         // Gradient loads (see ld_grad): plain with momentum; evict-first in the run-time-M kernel
         // without momentum; in the unrolled kernels without momentum plain once the call reads
-        // kPlainFromBytes of gradients or more. Measured plain / evict-first, fp32, isolated
+        // 1.5 GiB of gradients or more (launch option "plain_loads_from_mib"). Measured plain /
+        // evict-first, fp32, isolated
         // launches: M = 15: 1.02 at d = 2^24 (1.0 GB), 1.00 at 25.6 M (1.5 GB), 0.97 at 2^26, 0.96
         // at 2^28; M = 7: 1.05 at 2^24 (0.5 GB), 0.97 at 2^26 (1.9 GB) and at 61 M; M = 3: 1.13 at
         // 2^24, 1.02 at 2^26 (0.8 GB), 0.95 at 2^28 (3.2 GB).
         bool plain = MOM;
         if constexpr (!MOM && M_CT > 0)
-            plain = static_cast<int64_t>(s.M) * s.d * GT::kBytes >= kPlainFromBytes;
+            plain = static_cast<int64_t>(s.M) * s.d * GT::kBytes >= launch_plain_loads_from_bytes();
         if constexpr (MOM) {
             step_vec_kernel<M_CT, GT, MOM, APPLY, SEG, true><<<grid, threads, 0, st>>>(a);
         } else if constexpr (M_CT == 0) {

@@ -533,6 +533,22 @@ def test_results_do_not_depend_on_the_launch_shape(threads, blocks_per_sm):
         B.ss_set_launch_option("blocks_per_sm", 0)
 
 
+@pytest.mark.parametrize("from_mib", [1, 1 << 20], ids=["plain-gradient-loads", "evict-first-gradient-loads"])
+def test_results_do_not_depend_on_the_gradient_load_policy(from_mib):
+    """The unrolled kernels without momentum exist twice, with plain and with evict-first gradient
+    loads, chosen by the size of the call; the option forces either one at a size the oracle can check."""
+    try:
+        B.ss_set_launch_option("plain_loads_from_mib", from_mib)
+        d = 32 * 4096 * 9 + 8                                  # 4.7 MB per fp32 worker
+        for M in (1, 3, 7, 15, 16):
+            _fused_case(M, d, torch.float32, False, 0b1 if M > 2 else 0, 0.0, 0, steps=1, seed=4000 + M)
+        _fused_case(7, d, torch.bfloat16, False, 0, 0.0, 4, steps=1, seed=4100)    # 8-byte aligned bf16: quad form
+        _fused_case(15, d, torch.bfloat16, False, 0, 0.02, 0, steps=1, seed=4101)  # octet form
+        _fused_case(15, d, torch.float32, True, 0, 0.0, 0, steps=1, seed=4102)     # momentum: unaffected
+    finally:
+        B.ss_set_launch_option("plain_loads_from_mib", 0)
+
+
 def test_two_streams_run_independent_steps_side_by_side():
     """The library keeps no state between calls, so steps on different streams and buffers may
     overlap on the GPU."""

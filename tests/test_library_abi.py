@@ -184,6 +184,10 @@ def test_launch_option_validation(L):
     assert L.ss_set_launch_option(b"threads", 1024) == B.SS_ERR_INVALID_ARG
     assert L.ss_set_launch_option(b"threads", 256) == B.SS_OK
     assert L.ss_set_launch_option(b"blocks_per_sm", 4097) == B.SS_ERR_INVALID_ARG
+    assert L.ss_set_launch_option(b"plain_loads_from_mib", -1) == B.SS_ERR_INVALID_ARG
+    assert L.ss_set_launch_option(b"plain_loads_from_mib", (1 << 20) + 1) == B.SS_ERR_INVALID_ARG
+    assert L.ss_set_launch_option(b"plain_loads_from_mib", 1) == B.SS_OK
+    assert L.ss_set_launch_option(b"plain_loads_from_mib", 0) == B.SS_OK
     assert L.ss_set_launch_option(b"nope", 1) == B.SS_ERR_INVALID_ARG
     assert L.ss_set_launch_option(None, 1) == B.SS_ERR_INVALID_ARG
     assert L.ss_set_launch_option(b"threads", 128) == B.SS_OK
