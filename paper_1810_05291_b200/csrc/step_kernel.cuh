@@ -167,8 +167,9 @@ step_vec_kernel(const __grid_constant__ StepArgs<StepShape<M_CT, MOM>::NP> a) {
     const uint32_t T = static_cast<uint32_t>(M + 1) >> 1;
     const bool has_wd = a.wd != 0.0f;
 
-    for (int64_t base = static_cast<int64_t>(blockIdx.x) * tile; base < n_quads;
-         base += static_cast<int64_t>(gridDim.x) * tile) {
+    // one tile; WHOLE: the tile lies inside the vector, so no access of it needs a bounds test
+    auto do_tile = [&](int64_t base, auto whole_tag) {
+        constexpr bool WHOLE = decltype(whole_tag)::value;
         int64_t q[U];
         bool ok[U];
         float4 xq[U];
@@ -176,7 +177,8 @@ step_vec_kernel(const __grid_constant__ StepArgs<StepShape<M_CT, MOM>::NP> a) {
 #pragma unroll
         for (int u = 0; u < U; ++u) {
             q[u] = base + static_cast<int64_t>(u) * blockDim.x + threadIdx.x;
-            ok[u] = q[u] < n_quads;  // uniform over each 8-lane group: n_quads is a multiple of 8
+            // uniform over each 8-lane group: n_quads is a multiple of 8
+            ok[u] = WHOLE ? true : q[u] < n_quads;
             cnt[u].clear();
             if (APPLY && ok[u]) xq[u] = ld_rmw(reinterpret_cast<const float4*>(a.x) + q[u]);
         }
@@ -239,6 +241,16 @@ step_vec_kernel(const __grid_constant__ StepArgs<StepShape<M_CT, MOM>::NP> a) {
             }
         }
         if (a.words != nullptr) store_words<U>(a.words, vote, base, n_quads, lane);
+    };
+
+    for (int64_t base = static_cast<int64_t>(blockIdx.x) * tile; base < n_quads;
+         base += static_cast<int64_t>(gridDim.x) * tile) {
+        // the unguarded body pays where the worker loop is unrolled; the one-worker and
+        // run-time-M kernels keep a single (guarded) body, which costs them fewer registers
+        if (M_CT >= 3 && base + tile <= n_quads)
+            do_tile(base, std::true_type{});
+        else
+            do_tile(base, std::false_type{});
     }
 
     // the ragged last word (d not a multiple of 32): one warp, ballot form, run-time worker loop
