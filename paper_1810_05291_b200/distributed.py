@@ -122,6 +122,8 @@ class MajorityVoteWorker:
     been enqueued -- the benchmark records a CUDA event there to split a step into kernel time
     and exchange time."""
 
+    STATUS_RING = 256                # flag-ordered push: steps whose wait status is kept on the device
+
     def __init__(self, param: torch.Tensor, beta: Optional[float], lr: float,
                  weight_decay: float = 0.0, mode: str = "allgather", group=None, world=None,
                  rank=None, collectives=None, kernels=None, on_phase=None):
@@ -145,6 +147,7 @@ class MajorityVoteWorker:
         self.barrier = None
         self.flags = None            # flag-ordered push: see set_flag_exchange
         self.epoch = 0
+        self.checked_epoch = 0       # flag-ordered push: last step that check() has passed
         self.on_phase = on_phase
         if mode == "push" and beta is None:
             raise ValueError("push mode carries the momentum kernel: use it with Signum (beta set)")
@@ -171,29 +174,46 @@ class MajorityVoteWorker:
         the parity of the step, world * W_pad words each); ``dests[parity][m]`` is the address
         (tensor or int) of this worker's slot in worker m's buffer of that parity;
         ``flag_dests[m]`` is worker m's flag array and ``flags_local`` this worker's own. After a
-        step whose wait ran out of time the update is skipped as a whole; ``check()`` tells.
+        step whose wait ran out of time the update is skipped as a whole; ``check()`` tells, for
+        every step since the last check.
         ``signal_with_wait``: raise the flag in the launch that waits (``ss_flags_signal_wait``, one
         launch fewer per step) instead of right after the push; only for workers whose ``finish``
         follows their own ``pack_local`` without waiting for other workers' calls on this host."""
         world = self.ex.world
         if len(recv_bufs) != 2 or len(dests) != 2 or any(len(x) != world for x in dests) or len(flag_dests) != world:
             raise ValueError("need two receive buffers, two lists of one destination per worker, one flag array per worker")
+        # one status word per step, in a ring: a step whose wait ran out stays on record until
+        # check() has looked at it (finish() calls check() itself before it reuses a word)
         self.flags = dict(recv=list(recv_bufs), dests=[list(dests[0]), list(dests[1])], flag_dests=list(flag_dests),
                           local=flags_local, timeout_ns=int(timeout_ns), fused=bool(signal_with_wait),
-                          status=torch.zeros(1, dtype=torch.int32, device=self.x.device))
+                          status=torch.zeros(self.STATUS_RING, dtype=torch.int32, device=self.x.device))
+        self.checked_epoch = self.epoch
+
+    def step_status(self) -> torch.Tensor:
+        """Flag-ordered push: the status word (a one-element view) of the current step."""
+        slot = self.epoch % self.STATUS_RING
+        return self.flags["status"][slot: slot + 1]
 
     def check(self) -> None:
-        """Flag-ordered push: waits for the stream and raises if the last wait ran out of time
-        (RuntimeError naming the lowest worker whose packed signs had not arrived)."""
+        """Flag-ordered push: waits for the stream and raises if the wait of any step since the
+        last successful check ran out of time (RuntimeError naming the first such step and the
+        lowest worker whose packed signs had not arrived). The parameter update of such a step was
+        skipped on this worker, so its replica no longer follows the others'."""
+        self._check_through(self.epoch)
+
+    def _check_through(self, last_epoch: int) -> None:
         if self.flags is None:
             return
         if self.x.is_cuda:
             torch.cuda.synchronize(self.x.device)
-        status = int(self.flags["status"].item())
-        if status != 0:
-            raise RuntimeError("majority vote step %d: the packed signs of worker %d did not arrive within "
-                               "%.3f s; the parameter update of that step was skipped"
-                               % (self.epoch, status - 1, self.flags["timeout_ns"] * 1e-9))
+        ring = self.flags["status"].tolist()
+        for epoch in range(self.checked_epoch + 1, last_epoch + 1):
+            status = ring[epoch % self.STATUS_RING]
+            if status != 0:
+                raise RuntimeError("majority vote step %d: the packed signs of worker %d did not arrive within "
+                                   "%.3f s; the parameter update of that step was skipped"
+                                   % (epoch, status - 1, self.flags["timeout_ns"] * 1e-9))
+        self.checked_epoch = last_epoch
 
     def connect_push(self, group=None, barrier: str = "collective", timeout_ns: int = 1_000_000_000) -> None:
         """push mode across GPUs: allocates the receive buffer in symmetric memory
@@ -289,15 +309,18 @@ class MajorityVoteWorker:
         B, ex = self.B, self.ex
         if ex.mode == "push" and self.flags is not None:
             fl = self.flags
+            if self.epoch - self.checked_epoch >= self.STATUS_RING:
+                self._check_through(self.epoch - 1)   # this step's word still holds an unchecked step's status
+            status = self.step_status()
             ex.gathered = fl["recv"][self.epoch & 1]
             if fl["fused"]:
                 B.ss_flags_signal_wait(fl["flag_dests"], ex.rank, fl["local"], ex.world, self.epoch,
-                                       fl["timeout_ns"], fl["status"], stream)
+                                       fl["timeout_ns"], status, stream)
             else:
-                B.ss_flags_wait(fl["local"], ex.world, self.epoch, fl["timeout_ns"], fl["status"], stream)
+                B.ss_flags_wait(fl["local"], ex.world, self.epoch, fl["timeout_ns"], status, stream)
             self._phase("exchange:wait")
             B.ss_vote_apply_guarded(ex.worker_rows(), self.x, self.lr, self.weight_decay, flip_mask,
-                                    self.vote, fl["status"], stream)
+                                    self.vote, status, stream)
             self._phase("kernel:vote_apply")
             return self.vote
         if ex.mode == "push":

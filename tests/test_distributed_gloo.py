@@ -305,6 +305,56 @@ def test_a_worker_that_leaves_is_detected_by_the_bounded_wait(tmp_path):
     assert unchanged == "1"                          # the update of the failed step was skipped as a whole
 
 
+def _local_flag_workers(world, d, timeout_ns):
+    """`world` workers in this process, wired to one another's buffers and flags, on the stand-in kernels."""
+    workers = [MajorityVoteWorker(torch.zeros(d), 0.9, 1e-3, 0.0, "push", world=world, rank=m,
+                                  kernels=OracleKernels()) for m in range(world)]
+    W_pad = workers[0].ex.W_pad
+    bufs = [[torch.zeros(world * W_pad, dtype=torch.int32) for _ in (0, 1)] for _ in range(world)]
+    flags = [torch.zeros(64, dtype=torch.int32) for _ in range(world)]
+    for m, w in enumerate(workers):
+        slot = lambda buf: buf[m * W_pad: m * W_pad + w.ex.W]
+        w.set_flag_exchange(bufs[m], [[slot(bufs[p][parity]) for p in range(world)] for parity in (0, 1)],
+                            flags, flags[m], timeout_ns)
+    return workers
+
+
+def test_a_timed_out_step_is_reported_by_a_later_check():
+    """Host logic of the status ring: worker 1 is late for step 1; worker 0 carries on, step 2 goes
+    through, and only then is its status looked at. The check names step 1; worker 1 has no complaint."""
+    d = 500
+    w0, w1 = _local_flag_workers(2, d, timeout_ns=5_000_000)
+    g = torch.from_numpy(np.random.default_rng(3).standard_normal(d).astype(np.float32))
+    w0.pack_local(g)
+    x_before = w0.x.clone()
+    w0.finish(0)                                           # times out: worker 1 has not pushed
+    assert torch.equal(w0.x, x_before)
+    w1.pack_local(g)
+    w1.finish(0)
+    for w in (w0, w1):
+        w.pack_local(g)
+    for w in (w0, w1):
+        w.finish(0)
+    assert int(w0.step_status()) == 0 and not torch.equal(w0.x, x_before)
+    with pytest.raises(RuntimeError, match="step 1: the packed signs of worker 1 did not arrive"):
+        w0.check()
+    w1.check()
+    assert w1.checked_epoch == 2 and w0.checked_epoch == 0
+
+
+def test_finish_checks_by_itself_before_reusing_a_status_word():
+    w = _local_flag_workers(1, 40, timeout_ns=1_000_000)[0]
+    g = torch.ones(40)
+    for _ in range(w.STATUS_RING + 2):
+        w.step(g)
+    assert w.checked_epoch >= 1 and w.epoch == w.STATUS_RING + 2
+    # a failure that is about to fall out of the ring is raised by finish() itself
+    w.flags["status"][(w.checked_epoch + 1) % w.STATUS_RING] = 1
+    with pytest.raises(RuntimeError, match="worker 0 did not arrive"):
+        for _ in range(w.STATUS_RING):
+            w.step(g)
+
+
 @pytest.mark.parametrize("d,world", [(1, 1), (1, 4), (31, 2), (32, 2), (33, 2), (1000, 3), (1024, 4),
                                      (25_557_032, 15), (61_100_840, 7)])
 def test_slices_partition_the_words(d, world):

@@ -227,7 +227,7 @@ def test_wait_runs_out_when_a_worker_never_signals():
     torch.cuda.synchronize()
     waited = time.monotonic() - t0
     assert 0.025 < waited < 2.0
-    assert int(w.flags["status"].item()) == 3                           # 1 + the missing worker
+    assert int(w.step_status().item()) == 3                             # 1 + the missing worker
     with pytest.raises(RuntimeError, match="worker 2 did not arrive"):
         w.check()
     assert np.array_equal(w.x.cpu().numpy().view(np.uint32), x0.view(np.uint32))   # nothing was updated
@@ -245,6 +245,40 @@ def test_wait_runs_out_when_a_worker_never_signals():
     want = oracle.fused_step(grads, ref_v, ref_x, 0.9, 1e-3)
     assert np.array_equal(w.vote.cpu().numpy().view(np.uint32), want)
     assert np.array_equal(w.x.cpu().numpy().view(np.uint32), ref_x.view(np.uint32))
+
+
+def test_a_step_that_timed_out_stays_on_record_until_it_is_checked():
+    """Worker 1 is late for step 1 only (made on the host); worker 0 goes on to step 2, which goes
+    through, and looks at its status only afterwards: the check must still name step 1."""
+    M, d = 2, 20_000
+    rng = np.random.default_rng(6)
+    x0 = rng.standard_normal(d).astype(np.float32)
+    workers = _flag_workers(M, d, x0, timeout_ns=20_000_000)
+    g = [torch.from_numpy(rng.standard_normal(d).astype(np.float32)).to(DEV) for _ in range(M)]
+    workers[0].pack_local(g[0])
+    workers[0].finish(0)                                   # step 1: worker 1 has not pushed
+    workers[1].pack_local(g[1])
+    workers[1].finish(0)
+    for w in workers:                                      # step 2: everybody takes part
+        w.pack_local(g[0])
+    for w in workers:
+        w.finish(0)
+    torch.cuda.synchronize()
+    assert int(workers[0].step_status().item()) == 0       # the last step's own word is clean
+    with pytest.raises(RuntimeError, match="step 1: the packed signs of worker 1 did not arrive"):
+        workers[0].check()
+    workers[1].check()                                     # worker 1 missed nothing
+
+
+def test_the_status_ring_is_checked_before_a_word_is_reused():
+    M, d = 1, 64
+    w = _flag_workers(M, d, np.zeros(d, dtype=np.float32), timeout_ns=1_000_000)[0]
+    g = torch.ones(d, device=DEV)
+    for _ in range(w.STATUS_RING + 3):
+        w.step(g)
+    assert w.epoch == w.STATUS_RING + 3 and w.checked_epoch >= 2    # finish() ran a check by itself
+    w.check()
+    assert w.checked_epoch == w.epoch
 
 
 def test_flag_epochs_compare_as_serial_numbers():
