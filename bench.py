@@ -43,10 +43,10 @@ NOMINAL_HBM_GBS = 8000.0
 # sources have changed since, the entry no longer describes the kernel that runs and
 # roofline.traffic is reported as null until the counters are taken again.
 NCU_DRAM_BYTES_PER_COORD = {
-    (15, 4, True): {"bytes_per_coord": (1.040248e9 + 488.92e6) / 8388608, "capture_d": 8388608,
-                    "sources": "f32", "source_hash": "ffa6f1f19a623537"},
-    (15, 2, True): {"bytes_per_coord": (788.573e6 + 482.90e6) / 8388608, "capture_d": 8388608,
-                    "sources": "bf16", "source_hash": "9dd20825053442f2"},
+    (15, 4, True): {"bytes_per_coord": (1.040224e9 + 487.41e6) / 8388608, "capture_d": 8388608,
+                    "sources": "f32", "source_hash": "54a1c01e5932fd89"},
+    (15, 2, True): {"bytes_per_coord": (788.586e6 + 483.21e6) / 8388608, "capture_d": 8388608,
+                    "sources": "bf16", "source_hash": "16344c2aad055820"},
 }
 KERNEL_SOURCES = {
     "f32": ("step_kernel.cuh", "bitslice.cuh", "common.cuh"),

@@ -15,6 +15,9 @@
 // a pointer is not 16-byte aligned.
 #pragma once
 
+#include <cuda_bf16.h>
+#include <string.h>
+
 #include <type_traits>
 
 #include "bitslice.cuh"
@@ -271,33 +274,40 @@ step_ballot_kernel(const __grid_constant__ StepArgs<StepShape<M_CT, MOM>::NP> a)
 
 // Sign packing of one gradient buffer (ss_sign_pack): a pure read stream, so the kernel is kept
 // as lean as the arithmetic allows. Quad form: a thread loads U quads (128-bit requests, all
-// issued before the first is used), turns each into a sign nibble, and an OR tree over the eight
-// lanes of a word (three shuffles) assembles the word, stored by the group's first lane. Measured
-// against a read-only kernel of the same shape it runs at the same rate. One block per tile.
+// issued before the first is used), turns each into a sign nibble, and store_words assembles the
+// words across the eight lanes that share one. Tiles that lie inside the vector run without
+// bounds tests. Measured against a read-only kernel of the same shape it runs at the same rate.
+// One block per tile.
+// quads (fp32) and octets (bf16) a thread of the packing kernels has in flight: with 8 the fp32
+// kernel streams at the rate of a read-only kernel at every size (with 4 it fell 13 % behind)
+constexpr int kPackQuads = 8;
+constexpr int kPackOctets = 8;
 template <typename GT, int U>
 __global__ void __launch_bounds__(256)
 pack_vec_kernel(const void* __restrict__ g, uint32_t* __restrict__ words, int64_t d) {
     const int lane = threadIdx.x & 31;
-    const int k = lane & 7;
     const int64_t n_quads = (d >> 5) << 3;  // quads lying in complete words
     const int64_t tile = static_cast<int64_t>(blockDim.x) * U;
-    for (int64_t base = static_cast<int64_t>(blockIdx.x) * tile; base < n_quads;
-         base += static_cast<int64_t>(gridDim.x) * tile) {
+    // one tile; WHOLE: it lies inside the vector and its loads need no bounds test
+    auto do_tile = [&](int64_t base, auto whole_tag) {
+        constexpr bool WHOLE = decltype(whole_tag)::value;
         float4 v[U];
 #pragma unroll
         for (int u = 0; u < U; ++u) {
             const int64_t q = base + static_cast<int64_t>(u) * blockDim.x + threadIdx.x;
-            v[u] = q < n_quads ? GT::load4(g, q) : make_float4(-1.f, -1.f, -1.f, -1.f);
+            v[u] = (WHOLE || q < n_quads) ? GT::load4(g, q) : make_float4(-1.f, -1.f, -1.f, -1.f);
         }
+        uint32_t nib[U];
 #pragma unroll
-        for (int u = 0; u < U; ++u) {
-            uint32_t w = sign_nibble(v[u]) << (4 * k);
-            w |= __shfl_xor_sync(0xFFFFFFFFu, w, 1);
-            w |= __shfl_xor_sync(0xFFFFFFFFu, w, 2);
-            w |= __shfl_xor_sync(0xFFFFFFFFu, w, 4);
-            const int64_t q = base + static_cast<int64_t>(u) * blockDim.x + threadIdx.x;
-            if (k == 0 && q < n_quads) words[q >> 3] = w;
-        }
+        for (int u = 0; u < U; ++u) nib[u] = sign_nibble(v[u]);
+        store_words<U>(words, nib, base, n_quads, lane);
+    };
+    for (int64_t base = static_cast<int64_t>(blockIdx.x) * tile; base < n_quads;
+         base += static_cast<int64_t>(gridDim.x) * tile) {
+        if (base + tile <= n_quads)
+            do_tile(base, std::true_type{});
+        else
+            do_tile(base, std::false_type{});
     }
     // the ragged last word (d not a multiple of 32): one warp, one coordinate per lane
     if ((d & 31) != 0 && blockIdx.x == 0 && threadIdx.x < 32) {
@@ -308,40 +318,76 @@ pack_vec_kernel(const void* __restrict__ g, uint32_t* __restrict__ words, int64_
     }
 }
 
-// bf16 gradients with a 16-byte aligned pointer: a lane owns an octet (8 consecutive
-// coordinates, one 128-bit request; 64-bit requests top out near half the HBM rate), four lanes
-// make a word, two shuffles assemble it.
+// Sign bits of the eight bf16 values of a 128-bit load, coordinate i in bit i. One paired
+// bf16 comparison per register gives an all-ones or all-zero half per value (by value: +-0 -> 1,
+// NaN -> 0, as sign_bit); each register's two halves are masked down to its two bit positions,
+// the four registers are OR-ed, and the upper half is folded onto the lower.
+__device__ __forceinline__ uint32_t sign_byte_bf16(const uint4& r) {
+    const uint32_t raw[4] = {r.x, r.y, r.z, r.w};
+    uint32_t t = 0u;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        __nv_bfloat162 pair;
+        memcpy(&pair, &raw[i], 4);
+        const uint32_t ge = __hge2_mask(pair, __float2bfloat162_rn(0.0f));
+        t |= ge & ((1u << (2 * i)) | (2u << (2 * i + 16)));
+    }
+    return (t | (t >> 16)) & 0xFFu;
+}
+
+// Packed words from per-thread sign bytes of octets. Four neighbouring lanes hold the four bytes
+// of one word (lane k of the group owns bits 8k..8k+7). For every four rows of the tile the 4 x 4
+// matrix of bytes held by a group is transposed across its lanes by a two-stage butterfly, after
+// which lane k holds the complete word of row 4h + k and stores it (2 shuffles per 4 words).
+// Every lane of the warp must call this; U is a multiple of 4.
+template <int U>
+__device__ __forceinline__ void store_words_oct(uint32_t* words, const uint32_t* byte, int64_t base,
+                                                int64_t n_oct, int lane) {
+    static_assert(U % 4 == 0, "rows are transposed four at a time");
+    const int k = lane & 3;
+#pragma unroll
+    for (int h = 0; h < U / 4; ++h) {
+        uint32_t r = byte[4 * h] | (byte[4 * h + 1] << 8) | (byte[4 * h + 2] << 16) | (byte[4 * h + 3] << 24);
+        uint32_t o = __shfl_xor_sync(0xFFFFFFFFu, r, 2);
+        r = (k & 2) ? ((r & 0xFFFF0000u) | (o >> 16)) : ((r & 0x0000FFFFu) | (o << 16));
+        o = __shfl_xor_sync(0xFFFFFFFFu, r, 1);
+        r = (k & 1) ? ((r & 0xFF00FF00u) | ((o & 0xFF00FF00u) >> 8))
+                    : ((r & 0x00FF00FFu) | ((o & 0x00FF00FFu) << 8));
+        const int64_t ok = base + static_cast<int64_t>(4 * h + k) * blockDim.x + threadIdx.x;
+        if (ok < n_oct) words[ok >> 2] = r;
+    }
+}
+
+// bf16 gradients with a 16-byte aligned pointer: a lane owns U octets (8 consecutive coordinates
+// each, one 128-bit request; 64-bit requests top out near half the HBM rate), all loads issued
+// before the first is used; four lanes make a word.
 template <int U>
 __global__ void __launch_bounds__(256)
 pack_oct_bf16_kernel(const void* __restrict__ g, uint32_t* __restrict__ words, int64_t d) {
     const int lane = threadIdx.x & 31;
-    const int k = lane & 3;
     const int64_t n_oct = (d >> 5) << 2;  // octets lying in complete words
     const int64_t tile = static_cast<int64_t>(blockDim.x) * U;
-    for (int64_t base = static_cast<int64_t>(blockIdx.x) * tile; base < n_oct;
-         base += static_cast<int64_t>(gridDim.x) * tile) {
+    // one tile; WHOLE: it lies inside the vector and its loads need no bounds test
+    auto do_tile = [&](int64_t base, auto whole_tag) {
+        constexpr bool WHOLE = decltype(whole_tag)::value;
         uint4 v[U];
 #pragma unroll
         for (int u = 0; u < U; ++u) {
             const int64_t o = base + static_cast<int64_t>(u) * blockDim.x + threadIdx.x;
-            v[u] = o < n_oct ? ld_stream(reinterpret_cast<const uint4*>(g) + o)
-                             : make_uint4(0x80008000u, 0x80008000u, 0x80008000u, 0x80008000u);
+            v[u] = (WHOLE || o < n_oct) ? ld_stream(reinterpret_cast<const uint4*>(g) + o)
+                                        : make_uint4(0xFFFFFFFFu, 0xFFFFFFFFu, 0xFFFFFFFFu, 0xFFFFFFFFu);
         }
+        uint32_t byte[U];
 #pragma unroll
-        for (int u = 0; u < U; ++u) {
-            const uint32_t r[4] = {v[u].x, v[u].y, v[u].z, v[u].w};
-            uint32_t b = 0u;
-#pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                b |= sign_bit(__uint_as_float(r[i] << 16)) << (2 * i);
-                b |= sign_bit(__uint_as_float(r[i] & 0xFFFF0000u)) << (2 * i + 1);
-            }
-            uint32_t w = b << (8 * k);
-            w |= __shfl_xor_sync(0xFFFFFFFFu, w, 1);
-            w |= __shfl_xor_sync(0xFFFFFFFFu, w, 2);
-            const int64_t o = base + static_cast<int64_t>(u) * blockDim.x + threadIdx.x;
-            if (k == 0 && o < n_oct) words[o >> 2] = w;
-        }
+        for (int u = 0; u < U; ++u) byte[u] = sign_byte_bf16(v[u]);
+        store_words_oct<U>(words, byte, base, n_oct, lane);
+    };
+    for (int64_t base = static_cast<int64_t>(blockIdx.x) * tile; base < n_oct;
+         base += static_cast<int64_t>(gridDim.x) * tile) {
+        if (base + tile <= n_oct)
+            do_tile(base, std::true_type{});
+        else
+            do_tile(base, std::false_type{});
     }
     if ((d & 31) != 0 && blockIdx.x == 0 && threadIdx.x < 32) {
         const int64_t c = ((d >> 5) << 5) + lane;
@@ -386,7 +432,7 @@ cudaError_t launch_pack(const StepDesc& s, cudaStream_t st) {
     int grid = 1;
     cudaError_t err;
     if (GT::kBytes == 2 && (reinterpret_cast<uintptr_t>(s.g[0]) & 15) == 0) {
-        constexpr int U = 4;
+        constexpr int U = kPackOctets;
         auto kernel = pack_oct_bf16_kernel<U>;
         const int64_t octets = (s.d >> 5) << 2;
         const int64_t tile = static_cast<int64_t>(threads) * U;
@@ -394,7 +440,7 @@ cudaError_t launch_pack(const StepDesc& s, cudaStream_t st) {
         if (err != cudaSuccess) return err;
         kernel<<<grid, threads, 0, st>>>(s.g[0], s.words, s.d);
     } else if (s.vec) {
-        constexpr int U = 4;
+        constexpr int U = kPackQuads;
         auto kernel = pack_vec_kernel<GT, U>;
         const int64_t quads = (s.d >> 5) << 3;
         const int64_t tile = static_cast<int64_t>(threads) * U;
