@@ -66,29 +66,45 @@ __device__ __forceinline__ uint32_t ternary_code(float g, uint32_t r, float gmax
 }
 
 // ---- ||g||_inf over the elements that are not NaN. Non-negative floats order like their bit
-// patterns, so the reduction is an unsigned integer maximum (warp reduce, then one atomic per
-// warp into a word that the launch has zeroed). --------------------------------------------------
+// patterns, so the reduction is an unsigned integer maximum (warp and block reduce, then at most
+// one atomic per block into a word that the launch has zeroed). --------------------------------------------------
 template <typename GT, bool VEC>
 __global__ void __launch_bounds__(256) absmax_kernel(const void* __restrict__ g, int64_t d, unsigned* out) {
     float m = 0.0f;
     const int64_t stride = static_cast<int64_t>(gridDim.x) * blockDim.x;
     const int64_t tid = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
     if constexpr (VEC) {
+        constexpr int U = 8;  // quads in flight per thread: a pure read stream wants them all issued first
         const int64_t n_quads = d >> 2;
-        for (int64_t q = tid; q < n_quads; q += 2 * stride) {  // two independent loads per pass
-            const float4 a = GT::load4(g, q);
-            const bool second = q + stride < n_quads;
-            const float4 b = second ? GT::load4(g, q + stride) : make_float4(0.f, 0.f, 0.f, 0.f);
-            m = fmaxf(m, fmaxf(fmaxf(fabsf(a.x), fabsf(a.y)), fmaxf(fabsf(a.z), fabsf(a.w))));
-            m = fmaxf(m, fmaxf(fmaxf(fabsf(b.x), fabsf(b.y)), fmaxf(fabsf(b.z), fabsf(b.w))));
+        const int64_t tile = static_cast<int64_t>(blockDim.x) * U;
+        for (int64_t base = static_cast<int64_t>(blockIdx.x) * tile; base < n_quads;
+             base += static_cast<int64_t>(gridDim.x) * tile) {
+            float4 v[U];
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                const int64_t q = base + static_cast<int64_t>(u) * blockDim.x + threadIdx.x;
+                v[u] = q < n_quads ? GT::load4(g, q) : make_float4(0.f, 0.f, 0.f, 0.f);
+            }
+#pragma unroll
+            for (int u = 0; u < U; ++u)
+                m = fmaxf(m, fmaxf(fmaxf(fabsf(v[u].x), fabsf(v[u].y)), fmaxf(fabsf(v[u].z), fabsf(v[u].w))));
         }
         if (tid < (d & 3)) m = fmaxf(m, fabsf(GT::load1(g, (n_quads << 2) + tid)));
     } else {
         for (int64_t c = tid; c < d; c += stride) m = fmaxf(m, fabsf(GT::load1(g, c)));
     }
-    // fmaxf drops a NaN operand, so m is a non-negative number (or +Inf)
-    const unsigned w = __reduce_max_sync(0xFFFFFFFFu, __float_as_uint(m));
-    if ((threadIdx.x & 31) == 0 && w != 0u) atomicMax(out, w);
+    // fmaxf drops a NaN operand, so m is a non-negative number (or +Inf). Warp maximum, then the
+    // block's through shared memory; the block touches the result word only if it would raise it
+    // (the word only ever grows, so a stale read can cause a needless atomic, never a missed one).
+    __shared__ unsigned warp_max[kMaxBlockThreads / 32];
+    unsigned w = __reduce_max_sync(0xFFFFFFFFu, __float_as_uint(m));
+    if ((threadIdx.x & 31) == 0) warp_max[threadIdx.x >> 5] = w;
+    __syncthreads();
+    if (threadIdx.x < 32) {
+        const int n_warps = (blockDim.x + 31) >> 5;
+        w = __reduce_max_sync(0xFFFFFFFFu, threadIdx.x < n_warps ? warp_max[threadIdx.x] : 0u);
+        if (threadIdx.x == 0 && w > __ldcg(out)) atomicMax(out, w);
+    }
 }
 
 // ---- packing: a thread owns a quad (one 128-bit gradient load, one generator block), makes the
@@ -138,28 +154,39 @@ ternary_pack_kernel(const void* __restrict__ g, int64_t d, const float* __restri
     }
 }
 
-// ---- decoding: out_c = scale * q_c -------------------------------------------------------------
+// ---- decoding: out_c = scale * q_c. A warp takes 32 code words (512 coordinates) per pass: one
+// coalesced load of a word per lane, then four rounds in which lane l fetches the word that holds
+// quad 32 j + l of the pass from the lane that loaded it and stores that quad, so every store
+// instruction of the warp covers 512 contiguous bytes. -----------------------------------------------
 template <bool VEC>
 __global__ void __launch_bounds__(256)
 ternary_unpack_kernel(const uint32_t* __restrict__ codes, int64_t d, const float* __restrict__ scale_dev,
                       float* __restrict__ out) {
     const float scale = __ldg(scale_dev);
-    const int64_t stride = static_cast<int64_t>(gridDim.x) * blockDim.x;
-    const int64_t n_quads = (d + 3) >> 2;
-    for (int64_t q = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x; q < n_quads; q += stride) {
-        const uint32_t byte = (__ldg(codes + (q >> 2)) >> (8 * (q & 3))) & 0xFFu;
-        float f[4];
+    const int lane = threadIdx.x & 31;
+    const int64_t n_words = (d + 15) >> 4;
+    const int64_t warps = (static_cast<int64_t>(gridDim.x) * blockDim.x) >> 5;
+    for (int64_t w0 = ((static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x) >> 5) << 5; w0 < n_words;
+         w0 += warps << 5) {
+        const uint32_t mine = w0 + lane < n_words ? __ldg(codes + w0 + lane) : 0u;
 #pragma unroll
-        for (int i = 0; i < 4; ++i) {
-            const uint32_t code = (byte >> (2 * i)) & 3u;
-            const float t = (code & 1u) ? ((code & 2u) ? -1.0f : 1.0f) : 0.0f;
-            f[i] = __fmul_rn(scale, t);
-        }
-        if (VEC && 4 * q + 3 < d) {
-            __stcs(reinterpret_cast<float4*>(out) + q, make_float4(f[0], f[1], f[2], f[3]));
-        } else {
-            for (int i = 0; i < 4; ++i)
-                if (4 * q + i < d) out[4 * q + i] = f[i];
+        for (int j = 0; j < 4; ++j) {
+            const uint32_t word = __shfl_sync(0xFFFFFFFFu, mine, 8 * j + (lane >> 2));
+            const int64_t q = (w0 << 2) + 32 * j + lane;
+            const uint32_t byte = (word >> (8 * (lane & 3))) & 0xFFu;
+            float f[4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const uint32_t code = (byte >> (2 * i)) & 3u;
+                const float t = (code & 1u) ? ((code & 2u) ? -1.0f : 1.0f) : 0.0f;
+                f[i] = __fmul_rn(scale, t);
+            }
+            if (VEC && 4 * q + 3 < d) {
+                __stcs(reinterpret_cast<float4*>(out) + q, make_float4(f[0], f[1], f[2], f[3]));
+            } else {
+                for (int i = 0; i < 4; ++i)
+                    if (4 * q + i < d) out[4 * q + i] = f[i];
+            }
         }
     }
 }
@@ -209,10 +236,12 @@ int ss_absmax(const void* grad, ss_dtype dt, int64_t d, float* absmax_dev, void*
     const int threads = launch_threads();
     int grid = 1;
     unsigned* out = reinterpret_cast<unsigned*>(absmax_dev);
-    const int64_t items = vec ? ((d >> 2) + 1) / 2 + 4 : d;
+    // the quad form takes tiles of 8 quads per thread (plus a block's worth for the ragged end)
+    const int64_t items = vec ? (d >> 2) / 8 + threads : d;
 #define SS_ABSMAX(GT, VEC)                                                        \
     do {                                                                          \
-        e = stream_grid(threads, items, 16, &grid);                               \
+        e = VEC ? pick_grid(absmax_kernel<GT, VEC>, threads, (items + threads - 1) / threads, &grid) \
+                : stream_grid(threads, items, 16, &grid);                         \
         if (e != cudaSuccess) return cuda_status_public(e);                       \
         absmax_kernel<GT, VEC><<<grid, threads, 0, st>>>(grad, d, out);           \
     } while (0)
@@ -268,8 +297,8 @@ int ss_ternary_unpack(const uint32_t* codes, int64_t d, const float* scale_dev, 
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
     const int threads = launch_threads();
     int grid = 1;
-    const int64_t quads = (d + 3) >> 2;
-    cudaError_t e = pick_grid(ternary_unpack_kernel<true>, threads, (quads + threads - 1) / threads, &grid);
+    const int64_t words = (d + 15) >> 4;  // one word per lane and pass
+    cudaError_t e = pick_grid(ternary_unpack_kernel<true>, threads, (words + threads - 1) / threads, &grid);
     if (e != cudaSuccess) return cuda_status_public(e);
     if (aligned_to(out, 16))
         ternary_unpack_kernel<true><<<grid, threads, 0, st>>>(codes, d, scale_dev, out);
