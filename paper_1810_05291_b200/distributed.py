@@ -120,13 +120,14 @@ class MajorityVoteWorker:
     tests pass a stand-in so that the order of kernels and collectives can be driven on CPU ranks.
     ``on_phase`` (optional) is called with a label after every kernel or collective of a step has
     been enqueued -- the benchmark records a CUDA event there to split a step into kernel time
-    and exchange time."""
+    and exchange time. ``layout`` (optional ``fusion.FlatLayout``): the parameter vector is a model's
+    tensors back to back, each updated with its own learning rate and weight decay."""
 
     STATUS_RING = 256                # flag-ordered push: steps whose wait status is kept on the device
 
     def __init__(self, param: torch.Tensor, beta: Optional[float], lr: float,
                  weight_decay: float = 0.0, mode: str = "allgather", group=None, world=None,
-                 rank=None, collectives=None, kernels=None, on_phase=None):
+                 rank=None, collectives=None, kernels=None, on_phase=None, layout=None):
         if kernels is None:
             from . import binding as kernels
             if not param.is_cuda:
@@ -149,8 +150,20 @@ class MajorityVoteWorker:
         self.epoch = 0
         self.checked_epoch = 0       # flag-ordered push: last step that check() has passed
         self.on_phase = on_phase
+        # a fusion.FlatLayout of the parameter vector: the update then takes each tensor's own
+        # learning rate and weight decay from its device table and lr / weight_decay are unused
+        self.layout = layout
+        if layout is not None and layout.d != self.d:
+            raise ValueError("the layout describes %d coordinates, the parameter vector has %d" % (layout.d, self.d))
         if mode == "push" and beta is None:
             raise ValueError("push mode carries the momentum kernel: use it with Signum (beta set)")
+
+    def _vote_apply(self, rows, flip_mask: int, stream) -> None:
+        if self.layout is not None:
+            self.B.ss_vote_apply_segments(rows, self.x, self.layout.segments_dev, self.layout.n_segments,
+                                          flip_mask, self.vote, stream)
+        else:
+            self.B.ss_vote_apply(rows, self.x, self.lr, self.weight_decay, flip_mask, self.vote, stream)
 
     def _phase(self, label: str) -> None:
         if self.on_phase is not None:
@@ -180,6 +193,8 @@ class MajorityVoteWorker:
         launch fewer per step) instead of right after the push; only for workers whose ``finish``
         follows their own ``pack_local`` without waiting for other workers' calls on this host."""
         world = self.ex.world
+        if self.layout is not None:
+            raise ValueError("the flag-ordered push has no per-tensor form of its guarded update")
         if len(recv_bufs) != 2 or len(dests) != 2 or any(len(x) != world for x in dests) or len(flag_dests) != world:
             raise ValueError("need two receive buffers, two lists of one destination per worker, one flag array per worker")
         # one status word per step, in a ring: a step whose wait ran out stays on record until
@@ -326,8 +341,7 @@ class MajorityVoteWorker:
         if ex.mode == "push":
             self.barrier()
             self._phase("exchange:barrier")
-            B.ss_vote_apply(ex.worker_rows(), self.x, self.lr, self.weight_decay, flip_mask,
-                            self.vote, stream)
+            self._vote_apply(ex.worker_rows(), flip_mask, stream)
             self._phase("kernel:vote_apply")
             self.barrier()
             self._phase("exchange:barrier")
@@ -335,13 +349,15 @@ class MajorityVoteWorker:
         if ex.mode == "allgather":
             ex.gather()
             self._phase("exchange:all_gather")
-            B.ss_vote_apply(ex.worker_rows(), self.x, self.lr, self.weight_decay, flip_mask,
-                            self.vote, stream)
+            self._vote_apply(ex.worker_rows(), flip_mask, stream)
             self._phase("kernel:vote_apply")
             return self.vote
         ex.gather_vote()
         self._phase("exchange:all_gather")
-        B.ss_apply_vote(self.x, ex.vote_words(), self.lr, self.weight_decay, stream)
+        if self.layout is not None:
+            B.ss_apply_vote_segments(self.x, ex.vote_words(), self.layout.segments_dev, self.layout.n_segments, stream)
+        else:
+            B.ss_apply_vote(self.x, ex.vote_words(), self.lr, self.weight_decay, stream)
         self._phase("kernel:apply")
         return ex.vote_words()
 

@@ -19,10 +19,13 @@ from . import binding as B
 
 class FlatLayout:
     def __init__(self, shapes: Sequence[Sequence[int]], lrs: Sequence[float],
-                 weight_decays: Sequence[float], device, align: int = 4):
+                 weight_decays: Sequence[float], device, align: int = 4, kernels=None):
         """``align``: every tensor starts at a multiple of this many coordinates (4 keeps fp32
         views 16-byte aligned; 1 packs them with no padding). Padding coordinates belong to the
-        tensor before them and take its hyper-parameters."""
+        tensor before them and take its hyper-parameters. ``kernels``: the object whose ``ss_*``
+        functions are called, by default the binding of the CUDA library (the host-side tests
+        pass a stand-in)."""
+        self.B = kernels if kernels is not None else B
         if not (len(shapes) == len(lrs) == len(weight_decays)) or len(shapes) == 0:
             raise ValueError("need one shape, lr and weight_decay per tensor")
         if align < 1:
@@ -37,14 +40,14 @@ class FlatLayout:
         self.d = at
         self.device = torch.device(device)
         self.n_segments = len(self.shapes)
-        self.segments_dev = B.segment_table(self.n_segments, self.device)
+        self.segments_dev = self.B.segment_table(self.n_segments, self.device)
         self.set_hyperparameters(lrs, weight_decays)
 
     def set_hyperparameters(self, lrs: Sequence[float], weight_decays: Sequence[float], stream=None) -> None:
         """(Re)writes the device table, e.g. when a learning-rate schedule moves."""
         self.lrs = [float(v) for v in lrs]
         self.weight_decays = [float(v) for v in weight_decays]
-        B.ss_segments_upload(self.begins, self.lrs, self.weight_decays, self.d, self.segments_dev, stream)
+        self.B.ss_segments_upload(self.begins, self.lrs, self.weight_decays, self.d, self.segments_dev, stream)
 
     def flat(self, dtype=torch.float32) -> torch.Tensor:
         return torch.zeros(self.d, dtype=dtype, device=self.device)
@@ -58,5 +61,5 @@ class FlatLayout:
     def step(self, grads, momenta, param, beta: float, flip_mask: int = 0, vote_words_out=None,
              stream=None) -> None:
         """One iteration of Algorithm 1 over the whole model in one launch."""
-        B.ss_fused_step_segments(grads, momenta, param, beta, self.segments_dev, self.n_segments,
+        self.B.ss_fused_step_segments(grads, momenta, param, beta, self.segments_dev, self.n_segments,
                                  flip_mask, vote_words_out, stream)

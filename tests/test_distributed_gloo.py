@@ -135,6 +135,48 @@ class OracleKernels:
             self._u32(vote_words_out)[:] = vote
 
 
+    # ---- a fused vector of several tensors: the "device table" is a dict on the host here
+    @staticmethod
+    def ss_packed_words(d):
+        return (int(d) + 31) // 32
+
+    @staticmethod
+    def segment_table(n, device):
+        return {}
+
+    def ss_segments_upload(self, begins, lrs, weight_decays, d, segments_dev, stream=None):
+        self.calls.append("ss_segments_upload")
+        segments_dev.update(begins=list(begins), lrs=list(lrs), wds=list(weight_decays))
+
+    def ss_fused_step_segments(self, grads, momenta, param, beta, segments_dev, n_segments, flip_mask=0,
+                               vote_words_out=None, stream=None):
+        self.calls.append("ss_fused_step_segments")
+        t = segments_dev
+        vote = oracle.fused_step_segments([self._f32(g) for g in grads],
+                                          None if momenta is None else [self._f32(v) for v in momenta],
+                                          self._f32(param), beta, t["begins"], t["lrs"], t["wds"], flip_mask)
+        if vote_words_out is not None:
+            self._u32(vote_words_out)[:] = vote
+
+    def _apply_segments(self, param, vote, segments_dev):
+        # one "worker" whose gradient carries the vote's signs: its lone vote is the vote
+        d = param.numel()
+        g = np.where(oracle.unpack(vote, d) > 0, 1.0, -1.0).astype(np.float32)
+        t = segments_dev
+        oracle.fused_step_segments([g], None, self._f32(param), 0.0, t["begins"], t["lrs"], t["wds"], 0)
+
+    def ss_vote_apply_segments(self, packed, param, segments_dev, n_segments, flip_mask=0, vote_words_out=None,
+                               stream=None):
+        self.calls.append("ss_vote_apply_segments")
+        vote = oracle.majority_vote([self._u32(p).copy() for p in packed], param.numel(), flip_mask)
+        self._apply_segments(param, vote, segments_dev)
+        if vote_words_out is not None:
+            self._u32(vote_words_out)[:] = vote
+
+    def ss_apply_vote_segments(self, param, vote_words, segments_dev, n_segments, stream=None):
+        self.calls.append("ss_apply_vote_segments")
+        self._apply_segments(param, self._u32(vote_words).copy(), segments_dev)
+
     # ---- flag-ordered exchange: the flags are words of shared memory that other processes write
     SS_MAX_WORKERS = 64
 
