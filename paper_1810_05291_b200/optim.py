@@ -34,12 +34,16 @@ class SignumVote(torch.optim.Optimizer):
 
     A parameter whose ``grad`` is ``None`` at ``step()`` votes with a zero gradient, i.e. +1 under
     the one-bit sign. ``zero_grad`` always zeroes in place: the gradients must stay views of the
-    flat buffer. ``kernels`` / ``collectives`` replace the CUDA binding and ``torch.distributed``
-    (the host-side tests drive the optimiser on CPU ranks that way)."""
+    flat buffer. ``mode`` is the layout of the exchange between the workers (``"allgather"``,
+    ``"sharded"``, or ``"push"``, which is connected over the process group at construction with
+    ``push_barrier`` = ``"collective"`` or ``"signal"``). ``exchange``: run the worker-and-exchange
+    path even in a group of one (default: only with more than one process). ``kernels`` /
+    ``collectives`` replace the CUDA binding and ``torch.distributed`` (the host-side tests drive
+    the optimiser on CPU ranks that way)."""
 
     def __init__(self, params, lr: float = 1e-4, momentum: Optional[float] = 0.9, weight_decay: float = 0.0,
                  mode: str = "allgather", group=None, world: Optional[int] = None, rank: Optional[int] = None,
-                 kernels=None, collectives=None):
+                 kernels=None, collectives=None, exchange: Optional[bool] = None, push_barrier: str = "collective"):
         if lr < 0.0 or weight_decay < 0.0 or (momentum is not None and not 0.0 <= momentum < 1.0):
             raise ValueError("need lr >= 0, weight_decay >= 0 and 0 <= momentum < 1 (or None)")
         super().__init__(params, dict(lr=lr, weight_decay=weight_decay))
@@ -80,11 +84,15 @@ class SignumVote(torch.optim.Optimizer):
         self._tensors = tensors
         self.vote = torch.zeros(self.B.ss_packed_words(self.layout.d), dtype=torch.int32, device=device)
         self.worker = None
-        if world > 1:
+        if world > 1 if exchange is None else exchange:
             self.worker = MajorityVoteWorker(self.flat_param, momentum, lr, weight_decay, mode, group, world, rank,
                                              collectives, kernels, layout=self.layout)
             if momentum is not None:
                 self.worker.momentum = self.flat_momentum
+            if mode == "push":
+                if push_barrier not in ("collective", "signal"):
+                    raise ValueError("push_barrier must be 'collective' or 'signal'")
+                self.worker.connect_push(group, barrier=push_barrier)
 
     def _hyperparameters(self):
         lrs, wds = [], []

@@ -199,3 +199,32 @@ def test_gpu_one_process_matches_the_oracle(beta):
             assert np.array_equal(_bits(opt.flat_momentum), ref_v[0].view(np.uint32))
         words = opt.vote.cpu().numpy().view(np.uint32)
         assert words.shape[0] == oracle.packed_words(opt.layout.d)
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("mode", ["allgather", "sharded", "push"])
+def test_gpu_worker_path_with_a_table_in_a_group_of_one(mode):
+    """The worker-and-exchange path of the optimiser on real kernels and real NCCL collectives with
+    nobody to talk to: momentum and packing, the exchange, vote and per-tensor update."""
+    os.environ["MASTER_ADDR"] = "127.0.0.1"
+    os.environ["MASTER_PORT"] = str(_free_port())
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(dev)
+    dist.init_process_group("nccl", rank=0, world_size=1, device_id=dev)
+    try:
+        model = _model(13, dev, width=61)
+        opt = SignumVote(_groups(model), momentum=0.9, mode=mode, exchange=True)
+        assert opt.worker is not None
+        ref_x = opt.flat_param.cpu().numpy().copy()
+        ref_v = [np.zeros_like(ref_x)]
+        for step in range(3):
+            opt.zero_grad()
+            _loss(model, step, 0, dev).backward()
+            g = opt.flat_grad.cpu().numpy().copy()
+            _reference_step(opt, [g], ref_x, ref_v, 0.9)
+            opt.step()
+            torch.cuda.synchronize()
+            assert np.array_equal(_bits(opt.flat_param), ref_x.view(np.uint32)), "step %d" % step
+            assert np.array_equal(_bits(opt.flat_momentum), ref_v[0].view(np.uint32))
+    finally:
+        dist.destroy_process_group()
