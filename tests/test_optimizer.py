@@ -134,6 +134,26 @@ def test_state_dict_round_trip_continues_bit_for_bit():
     assert all(torch.equal(a, b) for a, b in zip(xa, xb)) and all(torch.equal(a, b) for a, b in zip(va, vb))
 
 
+def test_the_optimiser_trains_a_small_model():
+    """Signum's fixed-size steps bring a student network's loss on a fixed teacher's outputs down
+    (Theorem 1's setting with M = 1: x <- x - eta sign(v))."""
+    teacher = _model(21)
+    student = _model(22)
+    opt = SignumVote(student.parameters(), lr=2e-3, momentum=0.9, kernels=OracleKernels())
+    g = torch.Generator().manual_seed(5)
+    a = torch.randn(256, 5, generator=g)
+    with torch.no_grad():
+        b = teacher(a)
+    losses = []
+    for _ in range(300):
+        opt.zero_grad()
+        loss = ((student(a) - b) ** 2).mean()
+        loss.backward()
+        opt.step()
+        losses.append(float(loss.detach()))
+    assert losses[-1] < 0.2 * losses[0]
+
+
 def test_bad_arguments_are_refused():
     model = _model(4)
     with pytest.raises(ValueError):
