@@ -265,6 +265,13 @@ int ss_vote_apply_segments(const uint32_t* const* packed, int M, int64_t d, uint
                            float* param, const ss_segment* segments_dev, int n_segments,
                            uint32_t* vote_words_out, void* cuda_stream);
 
+/* ss_vote_apply_guarded over a fused vector of tensors: ss_vote_apply_segments that does nothing
+ * at all when the word at skip_if_nonzero_dev is not zero. */
+int ss_vote_apply_guarded_segments(const uint32_t* const* packed, int M, int64_t d, uint64_t flip_mask,
+                                   float* param, const ss_segment* segments_dev, int n_segments,
+                                   uint32_t* vote_words_out, const uint32_t* skip_if_nonzero_dev,
+                                   void* cuda_stream);
+
 /* ss_apply_vote with per-tensor eta and lambda from a device segment table. */
 int ss_apply_vote_segments(float* param, const uint32_t* vote_words, int64_t d,
                            const ss_segment* segments_dev, int n_segments, void* cuda_stream);

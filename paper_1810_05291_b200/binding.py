@@ -38,7 +38,8 @@ EXPORTS = ("ss_packed_words", "ss_status_string", "ss_last_cuda_error", "ss_sign
            "ss_segments_upload", "ss_fused_step_segments", "ss_apply_vote_segments",
            "ss_vote_apply", "ss_vote_apply_segments", "ss_signum_update_push", "ss_vote_tally", "ss_fused_step_host", "ss_fused_step_host_static", "ss_set_launch_option",
            "ss_ternary_words", "ss_absmax", "ss_ternary_pack", "ss_ternary_unpack",
-           "ss_flags_signal", "ss_flags_wait", "ss_flags_signal_wait", "ss_vote_apply_guarded")
+           "ss_flags_signal", "ss_flags_wait", "ss_flags_signal_wait", "ss_vote_apply_guarded",
+           "ss_vote_apply_guarded_segments")
 
 
 class ss_segment(ctypes.Structure):
@@ -101,8 +102,10 @@ def lib() -> ctypes.CDLL:
     L.ss_flags_signal.argtypes = [vp, i32, i32, ctypes.c_uint32, vp]
     L.ss_flags_wait.argtypes = [vp, i32, ctypes.c_uint32, u64, vp, vp]
     L.ss_vote_apply_guarded.argtypes = [vp, i32, i64, u64, vp, f32, f32, vp, vp, vp]
+    L.ss_vote_apply_guarded_segments.argtypes = [vp, i32, i64, u64, vp, vp, i32, vp, vp, vp]
     L.ss_flags_signal_wait.argtypes = [vp, i32, i32, vp, i32, ctypes.c_uint32, u64, vp, vp]
-    for name in ("ss_flags_signal", "ss_flags_wait", "ss_flags_signal_wait", "ss_vote_apply_guarded"):
+    for name in ("ss_flags_signal", "ss_flags_wait", "ss_flags_signal_wait", "ss_vote_apply_guarded",
+                 "ss_vote_apply_guarded_segments"):
         getattr(L, name).restype = i32
     for name in ("ss_absmax", "ss_ternary_pack", "ss_ternary_unpack"):
         getattr(L, name).restype = i32
@@ -443,3 +446,17 @@ def ss_vote_apply_guarded(packed: Sequence[torch.Tensor], param: torch.Tensor, l
                                        _dev(param, torch.float32, "param"), float(lr), float(weight_decay),
                                        w_ptr, _dev(skip_if_nonzero_dev, torch.int32, "skip_if_nonzero_dev", 1),
                                        _stream(stream)), "ss_vote_apply_guarded")
+
+
+def ss_vote_apply_guarded_segments(packed: Sequence[torch.Tensor], param: torch.Tensor,
+                                   segments_dev: torch.Tensor, n_segments: int, flip_mask: int,
+                                   vote_words_out: Optional[torch.Tensor], skip_if_nonzero_dev: torch.Tensor,
+                                   stream=None) -> None:
+    d = param.numel()
+    ptrs = [_words(p, d, "packed[%d]" % m) for m, p in enumerate(packed)]
+    w_ptr = None if vote_words_out is None else _words(vote_words_out, d, "vote_words_out")
+    _check(lib().ss_vote_apply_guarded_segments(_ptr_array(ptrs), len(ptrs), d, int(flip_mask),
+                                                _dev(param, torch.float32, "param"),
+                                                _segments(segments_dev, n_segments), int(n_segments), w_ptr,
+                                                _dev(skip_if_nonzero_dev, torch.int32, "skip_if_nonzero_dev", 1),
+                                                _stream(stream)), "ss_vote_apply_guarded_segments")

@@ -317,19 +317,37 @@ static int vote_apply_common(const uint32_t* const* packed, int M, int64_t d, ui
                                                  static_cast<cudaStream_t>(cuda_stream)));
 }
 
+// the guard word is read while the call writes: it may lie in neither output
+static int guard_ok(const uint32_t* guard, int64_t d, const float* param, const uint32_t* vote_words_out) {
+    if (guard == nullptr) return SS_ERR_INVALID_ARG;
+    if (!aligned(guard, 4)) return SS_ERR_MISALIGNED;
+    if (d > 0 && d_ok(d)) {
+        if (param != nullptr && overlap(guard, 4, param, static_cast<size_t>(d) * 4)) return SS_ERR_INVALID_ARG;
+        if (vote_words_out != nullptr && overlap(guard, 4, vote_words_out, static_cast<size_t>((d + 31) / 32) * 4))
+            return SS_ERR_INVALID_ARG;
+    }
+    return SS_OK;
+}
+
 int ss_vote_apply_guarded(const uint32_t* const* packed, int M, int64_t d, uint64_t flip_mask,
                           float* param, float lr, float weight_decay, uint32_t* vote_words_out,
                           const uint32_t* skip_if_nonzero_dev, void* cuda_stream) {
-    if (skip_if_nonzero_dev == nullptr) return SS_ERR_INVALID_ARG;
-    if (!aligned(skip_if_nonzero_dev, 4)) return SS_ERR_MISALIGNED;
-    if (d > 0 && d_ok(d)) {  // the guard word is read while the call writes: it may lie in neither output
-        if (param != nullptr && overlap(skip_if_nonzero_dev, 4, param, static_cast<size_t>(d) * 4))
-            return SS_ERR_INVALID_ARG;
-        if (vote_words_out != nullptr &&
-            overlap(skip_if_nonzero_dev, 4, vote_words_out, static_cast<size_t>((d + 31) / 32) * 4))
-            return SS_ERR_INVALID_ARG;
-    }
+    const int rc = guard_ok(skip_if_nonzero_dev, d, param, vote_words_out);
+    if (rc != SS_OK) return rc;
     return vote_apply_common(packed, M, d, flip_mask, param, lr, weight_decay, nullptr, 0,
+                             vote_words_out, cuda_stream, skip_if_nonzero_dev);
+}
+
+int ss_vote_apply_guarded_segments(const uint32_t* const* packed, int M, int64_t d, uint64_t flip_mask,
+                                   float* param, const ss_segment* segments_dev, int n_segments,
+                                   uint32_t* vote_words_out, const uint32_t* skip_if_nonzero_dev,
+                                   void* cuda_stream) {
+    const int rc = guard_ok(skip_if_nonzero_dev, d, param, vote_words_out);
+    if (rc != SS_OK) return rc;
+    if (n_segments < 1) return SS_ERR_INVALID_ARG;
+    if (d > 0 && segments_dev == nullptr) return SS_ERR_INVALID_ARG;
+    if (d > 0 && !aligned(segments_dev, 8)) return SS_ERR_MISALIGNED;
+    return vote_apply_common(packed, M, d, flip_mask, param, 0.0f, 0.0f, segments_dev, n_segments,
                              vote_words_out, cuda_stream, skip_if_nonzero_dev);
 }
 

@@ -193,8 +193,6 @@ class MajorityVoteWorker:
         launch fewer per step) instead of right after the push; only for workers whose ``finish``
         follows their own ``pack_local`` without waiting for other workers' calls on this host."""
         world = self.ex.world
-        if self.layout is not None:
-            raise ValueError("the flag-ordered push has no per-tensor form of its guarded update")
         if len(recv_bufs) != 2 or len(dests) != 2 or any(len(x) != world for x in dests) or len(flag_dests) != world:
             raise ValueError("need two receive buffers, two lists of one destination per worker, one flag array per worker")
         # one status word per step, in a ring: a step whose wait ran out stays on record until
@@ -334,8 +332,12 @@ class MajorityVoteWorker:
             else:
                 B.ss_flags_wait(fl["local"], ex.world, self.epoch, fl["timeout_ns"], status, stream)
             self._phase("exchange:wait")
-            B.ss_vote_apply_guarded(ex.worker_rows(), self.x, self.lr, self.weight_decay, flip_mask,
-                                    self.vote, status, stream)
+            if self.layout is not None:
+                B.ss_vote_apply_guarded_segments(ex.worker_rows(), self.x, self.layout.segments_dev,
+                                                 self.layout.n_segments, flip_mask, self.vote, status, stream)
+            else:
+                B.ss_vote_apply_guarded(ex.worker_rows(), self.x, self.lr, self.weight_decay, flip_mask,
+                                        self.vote, status, stream)
             self._phase("kernel:vote_apply")
             return self.vote
         if ex.mode == "push":

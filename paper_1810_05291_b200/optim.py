@@ -36,7 +36,8 @@ class SignumVote(torch.optim.Optimizer):
     the one-bit sign. ``zero_grad`` always zeroes in place: the gradients must stay views of the
     flat buffer. ``mode`` is the layout of the exchange between the workers (``"allgather"``,
     ``"sharded"``, or ``"push"``, which is connected over the process group at construction with
-    ``push_barrier`` = ``"collective"`` or ``"signal"``). ``exchange``: run the worker-and-exchange
+    ``push_barrier`` = ``"collective"``, ``"signal"`` or ``"flags"``; with ``"flags"`` call
+    ``opt.worker.check()`` to learn of a step that a missing worker made this one skip). ``exchange``: run the worker-and-exchange
     path even in a group of one (default: only with more than one process). ``kernels`` /
     ``collectives`` replace the CUDA binding and ``torch.distributed`` (the host-side tests drive
     the optimiser on CPU ranks that way)."""
@@ -90,8 +91,8 @@ class SignumVote(torch.optim.Optimizer):
             if momentum is not None:
                 self.worker.momentum = self.flat_momentum
             if mode == "push":
-                if push_barrier not in ("collective", "signal"):
-                    raise ValueError("push_barrier must be 'collective' or 'signal'")
+                if push_barrier not in ("collective", "signal", "flags"):
+                    raise ValueError("push_barrier must be 'collective', 'signal' or 'flags'")
                 self.worker.connect_push(group, barrier=push_barrier)
 
     def _hyperparameters(self):

@@ -212,6 +212,15 @@ class OracleKernels:
         self.ss_vote_apply(packed, param, lr, weight_decay, flip_mask, vote_words_out, stream)
         self.calls[-1] = "ss_vote_apply_guarded"
 
+    def ss_vote_apply_guarded_segments(self, packed, param, segments_dev, n_segments, flip_mask, vote_words_out,
+                                       skip_if_nonzero_dev, stream=None):
+        self.calls.append("ss_vote_apply_guarded_segments")
+        if int(skip_if_nonzero_dev[0]) != 0:
+            return
+        self.calls.pop()
+        self.ss_vote_apply_segments(packed, param, segments_dev, n_segments, flip_mask, vote_words_out, stream)
+        self.calls[-1] = "ss_vote_apply_guarded_segments"
+
 
 EXPECTED_ORDER = {
     "allgather": ["start", "kernel:pack", "exchange:all_gather", "kernel:vote_apply"],

@@ -318,6 +318,36 @@ def test_guarded_vote_apply_skips_everything_or_nothing():
         assert torch.equal(xs, xr) and torch.equal(vote, vr)
 
 
+def test_guarded_vote_apply_over_a_table_of_tensors():
+    from paper_1810_05291_b200 import binding as B
+    from paper_1810_05291_b200.fusion import FlatLayout
+    M = 5
+    layout = FlatLayout([(37, 11), (5,), (1000,), (3, 3, 7)], [1e-2, 3e-3, 1e-3, 2e-2], [0.0, 0.01, 0.1, 0.0], DEV)
+    d = layout.d
+    gen = torch.Generator(device=DEV).manual_seed(9)
+    W = B.ss_packed_words(d)
+    packed = [torch.randint(-(1 << 31), 1 << 31, (W,), generator=gen, device=DEV, dtype=torch.int64).to(torch.int32)
+              for _ in range(M)]
+    x0 = torch.randn(d, generator=gen, device=DEV)
+    xs = x0.clone()
+    vote = torch.full((W,), -1, dtype=torch.int32, device=DEV)
+    guard = torch.full((1,), 2, dtype=torch.int32, device=DEV)
+    B.ss_vote_apply_guarded_segments(packed, xs, layout.segments_dev, layout.n_segments, 0b100, vote, guard)
+    assert torch.equal(xs, x0) and bool((vote == -1).all())
+    guard.zero_()
+    B.ss_vote_apply_guarded_segments(packed, xs, layout.segments_dev, layout.n_segments, 0b100, vote, guard)
+    xr, vr = x0.clone(), torch.zeros(W, dtype=torch.int32, device=DEV)
+    B.ss_vote_apply_segments(packed, xr, layout.segments_dev, layout.n_segments, 0b100, vr)
+    assert torch.equal(xs, xr) and torch.equal(vote, vr)
+    # against the oracle: the vote, then the per-tensor update (a lone worker whose gradient carries the vote's signs)
+    want_vote = oracle.majority_vote([p.cpu().numpy().view(np.uint32) for p in packed], d, 0b100)
+    assert np.array_equal(vote.cpu().numpy().view(np.uint32), want_vote)
+    ref = x0.cpu().numpy().copy()
+    g = np.where(oracle.unpack(want_vote, d) > 0, 1.0, -1.0).astype(np.float32)
+    oracle.fused_step_segments([g], None, ref, 0.0, layout.begins, layout.lrs, layout.weight_decays, 0)
+    assert np.array_equal(xs.cpu().numpy().view(np.uint32), ref.view(np.uint32))
+
+
 def _nccl_worker(rank, world, port, mode, d, beta, flip, errors):
     """One process = one worker of Algorithm 1 on GPU `rank`, talking NCCL to the others."""
     os.environ["MASTER_ADDR"] = "127.0.0.1"

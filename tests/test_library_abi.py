@@ -176,6 +176,13 @@ def test_flag_exchange_argument_errors(L):
     assert L.ss_vote_apply_guarded(arr, 2, 64, 0, vp(0x70000), 0.1, 0.0, None, vp(0x9001), None) == B.SS_ERR_MISALIGNED
     assert L.ss_vote_apply_guarded(arr, 2, 64, 0, vp(0x70000), 0.1, 0.0, None, vp(0x70010), None) == B.SS_ERR_INVALID_ARG  # guard inside param
     assert L.ss_vote_apply_guarded(arr, 2, 64, 0, vp(0x70000), 0.1, 0.0, vp(0x80000), vp(0x80004), None) == B.SS_ERR_INVALID_ARG  # guard inside the vote
+    seg = vp(0x90000)
+    assert L.ss_vote_apply_guarded_segments(arr, 2, 64, 0, vp(0x70000), seg, 1, None, None, None) == B.SS_ERR_INVALID_ARG
+    assert L.ss_vote_apply_guarded_segments(arr, 2, 64, 0, vp(0x70000), seg, 1, None, vp(0x9001), None) == B.SS_ERR_MISALIGNED
+    assert L.ss_vote_apply_guarded_segments(arr, 2, 64, 0, vp(0x70000), seg, 1, None, vp(0x70010), None) == B.SS_ERR_INVALID_ARG
+    assert L.ss_vote_apply_guarded_segments(arr, 2, 64, 0, vp(0x70000), seg, 0, None, vp(0xA0000), None) == B.SS_ERR_INVALID_ARG  # empty table
+    assert L.ss_vote_apply_guarded_segments(arr, 2, 64, 0, vp(0x70000), None, 1, None, vp(0xA0000), None) == B.SS_ERR_INVALID_ARG
+    assert L.ss_vote_apply_guarded_segments(arr, 2, 64, 0, vp(0x70000), vp(0x90004), 1, None, vp(0xA0000), None) == B.SS_ERR_MISALIGNED
 
 
 def test_launch_option_validation(L):

@@ -222,7 +222,7 @@ def test_gpu_one_process_matches_the_oracle(beta):
 
 
 @pytest.mark.gpu
-@pytest.mark.parametrize("mode", ["allgather", "sharded", "push"])
+@pytest.mark.parametrize("mode", ["allgather", "sharded", "push", "push:signal", "push:flags"])
 def test_gpu_worker_path_with_a_table_in_a_group_of_one(mode):
     """The worker-and-exchange path of the optimiser on real kernels and real NCCL collectives with
     nobody to talk to: momentum and packing, the exchange, vote and per-tensor update."""
@@ -233,7 +233,8 @@ def test_gpu_worker_path_with_a_table_in_a_group_of_one(mode):
     dist.init_process_group("nccl", rank=0, world_size=1, device_id=dev)
     try:
         model = _model(13, dev, width=61)
-        opt = SignumVote(_groups(model), momentum=0.9, mode=mode, exchange=True)
+        layout, _, barrier = mode.partition(":")
+        opt = SignumVote(_groups(model), momentum=0.9, mode=layout, exchange=True, push_barrier=barrier or "collective")
         assert opt.worker is not None
         ref_x = opt.flat_param.cpu().numpy().copy()
         ref_v = [np.zeros_like(ref_x)]
@@ -244,6 +245,7 @@ def test_gpu_worker_path_with_a_table_in_a_group_of_one(mode):
             _reference_step(opt, [g], ref_x, ref_v, 0.9)
             opt.step()
             torch.cuda.synchronize()
+            opt.worker.check()
             assert np.array_equal(_bits(opt.flat_param), ref_x.view(np.uint32)), "step %d" % step
             assert np.array_equal(_bits(opt.flat_momentum), ref_v[0].view(np.uint32))
     finally:
